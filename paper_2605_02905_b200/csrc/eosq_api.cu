@@ -1,0 +1,386 @@
+// C-ABI entry points of the eosq library: argument checks, the context's cached constants,
+// workspace carving and the launch sequence of each call.
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+
+#include "eosq_common.cuh"
+
+using namespace eosq;
+
+namespace {
+
+bool record_cuda(eosq_ctx *ctx, cudaError_t err, const char *what) {
+    if (err == cudaSuccess) return false;
+    if (ctx) ctx->last_error = std::string(what) + ": " + cudaGetErrorString(err);
+    return true;
+}
+
+int check_shape(int n, int d, int bits) {
+    if (d != D || bits < 1 || bits > 4 || n < d || n > NMAX || (n % 8) != 0) return EOSQ_ERR_UNSUPPORTED;
+    return EOSQ_OK;
+}
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Carve the scratch arrays of one chunk (capacity `cap` blocks) out of `base`.
+size_t carve(void *base, int64_t cap, Workspace *ws) {
+    char *p = static_cast<char *>(base);
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        void *q = p ? p + off : nullptr;
+        off = align_up(off + bytes, 256);
+        return q;
+    };
+    Workspace w;
+    w.gram = static_cast<double *>(take(sizeof(double) * cap * D * D));
+    w.diag = static_cast<double *>(take(sizeof(double) * cap * D));
+    w.off = static_cast<double *>(take(sizeof(double) * cap * D));
+    w.tau = static_cast<double *>(take(sizeof(double) * cap * D));
+    w.lam = static_cast<double *>(take(sizeof(double) * cap * D));
+    w.vr = static_cast<float *>(take(sizeof(float) * cap * RMAX * D));
+    w.coef = static_cast<float *>(take(sizeof(float) * cap * RMAX));
+    w.rank = static_cast<int *>(take(sizeof(int) * cap));
+    if (ws) *ws = w;
+    return off;
+}
+
+int get_rotation(eosq_ctx *ctx, int d, uint64_t seed, Rotation *out) {
+    for (const Rotation &r : ctx->rotations)
+        if (r.seed == seed) {
+            *out = r;
+            return EOSQ_OK;
+        }
+    std::vector<double> pi(static_cast<size_t>(d) * d);
+    int rc = eosq_rotation(d, seed, pi.data());
+    if (rc != EOSQ_OK) return rc;
+    std::vector<float> f(pi.size()), ft(pi.size());
+    for (int c = 0; c < d; ++c)
+        for (int j = 0; j < d; ++j) {
+            f[static_cast<size_t>(c) * d + j] = static_cast<float>(pi[static_cast<size_t>(c) * d + j]);
+            ft[static_cast<size_t>(j) * d + c] = static_cast<float>(pi[static_cast<size_t>(c) * d + j]);
+        }
+    Rotation r;
+    r.seed = seed;
+    const size_t bytes = sizeof(float) * f.size();
+    if (record_cuda(ctx, cudaMalloc(&r.pi, bytes), "cudaMalloc(rotation)")) return EOSQ_ERR_CUDA;
+    if (record_cuda(ctx, cudaMalloc(&r.pi_t, bytes), "cudaMalloc(rotation)")) return EOSQ_ERR_CUDA;
+    if (record_cuda(ctx, cudaMemcpy(r.pi, f.data(), bytes, cudaMemcpyHostToDevice), "cudaMemcpy(rotation)")) return EOSQ_ERR_CUDA;
+    if (record_cuda(ctx, cudaMemcpy(r.pi_t, ft.data(), bytes, cudaMemcpyHostToDevice), "cudaMemcpy(rotation)")) return EOSQ_ERR_CUDA;
+    ctx->rotations.push_back(r);
+    *out = r;
+    return EOSQ_OK;
+}
+
+int get_codebook(int d, int bits, Codebook *cb) {
+    double cen[16], thr[15];
+    int rc = eosq_codebook(bits, d, cen, thr);
+    if (rc != EOSQ_OK) return rc;
+    std::memset(cb, 0, sizeof(*cb));
+    cb->bits = bits;
+    for (int i = 0; i < (1 << bits); ++i) cb->centroid[i] = static_cast<float>(cen[i]);
+    for (int i = 0; i + 1 < (1 << bits); ++i) cb->threshold[i] = static_cast<float>(thr[i]);
+    return EOSQ_OK;
+}
+
+// Offset every array of a cache by `b0` blocks (so kernels can index from 0 within a chunk).
+eosq_cache_t shifted(const eosq_cache_t &c, int64_t b0, int n, int bits) {
+    eosq_cache_t o = c;
+    const int64_t rb = D * bits / 8;
+    if (o.codes) o.codes += b0 * n * rb;
+    if (o.norms) o.norms += b0 * n;
+    if (o.rank) o.rank += b0;
+    if (o.sigma) o.sigma += b0 * RMAX;
+    if (o.phi) o.phi += b0 * RMAX;
+    if (o.P) o.P += b0 * RMAX * n;
+    if (o.V) o.V += b0 * RMAX * D;
+    if (o.status) o.status += b0;
+    if (o.eig) o.eig += b0 * D;
+    if (o.lambda_plus) o.lambda_plus += b0;
+    if (o.vr32) o.vr32 += b0 * RMAX * D;
+    if (o.coef) o.coef += b0 * RMAX;
+    return o;
+}
+
+cudaEvent_t take_event(eosq_ctx *ctx) {
+    if (!ctx->free_events.empty()) {
+        cudaEvent_t e = ctx->free_events.back();
+        ctx->free_events.pop_back();
+        return e;
+    }
+    cudaEvent_t e = nullptr;
+    cudaEventCreate(&e);
+    return e;
+}
+
+// Runs `launch` (which enqueues exactly one kernel on `s`), counting it and, when profiling is
+// on, bracketing it with events.
+template <typename F>
+void run_stage(eosq_ctx *ctx, int stage, cudaStream_t s, F &&launch) {
+    if (ctx->profile) {
+        eosq_ctx::Timed t{stage, take_event(ctx), take_event(ctx)};
+        cudaEventRecord(t.start, s);
+        launch();
+        cudaEventRecord(t.stop, s);
+        ctx->timed.push_back(t);
+    } else {
+        launch();
+    }
+    ctx->launches += 1;
+}
+
+bool cache_required_ok(const eosq_cache_t *c) {
+    return c && c->codes && c->norms && c->rank && c->sigma && c->phi && c->P && c->V && c->status;
+}
+
+}  // namespace
+
+extern "C" size_t eosq_workspace_bytes(int64_t num_blocks, int n, int d) {
+    (void)n;
+    if (num_blocks <= 0 || d != D) return 0;
+    return carve(nullptr, std::min<int64_t>(num_blocks, CHUNK_BLOCKS), nullptr);
+}
+
+extern "C" int eosq_create(eosq_ctx **out) {
+    if (!out) return EOSQ_ERR_INVALID_ARG;
+    if (eosq_pilot_k(D) != KPILOT) return EOSQ_ERR_UNSUPPORTED;
+    eosq_ctx *ctx = new (std::nothrow) eosq_ctx();
+    if (!ctx) return EOSQ_ERR_INVALID_ARG;
+    if (record_cuda(ctx, cudaGetDevice(&ctx->device), "cudaGetDevice")) {
+        delete ctx;
+        return EOSQ_ERR_CUDA;
+    }
+    *out = ctx;
+    return EOSQ_OK;
+}
+
+extern "C" int eosq_destroy(eosq_ctx *ctx) {
+    if (!ctx) return EOSQ_OK;
+    for (Rotation &r : ctx->rotations) {
+        cudaFree(r.pi);
+        cudaFree(r.pi_t);
+    }
+    for (eosq_ctx::Timed &t : ctx->timed) {
+        cudaEventDestroy(t.start);
+        cudaEventDestroy(t.stop);
+    }
+    for (cudaEvent_t e : ctx->free_events) cudaEventDestroy(e);
+    delete ctx;
+    return EOSQ_OK;
+}
+
+extern "C" int eosq_profile_enable(eosq_ctx *ctx, int on) {
+    if (!ctx) return EOSQ_ERR_INVALID_ARG;
+    ctx->profile = on != 0;
+    return EOSQ_OK;
+}
+
+extern "C" int eosq_profile_read(eosq_ctx *ctx, float *ms, int64_t *launches) {
+    if (!ctx || !ms || !launches) return EOSQ_ERR_INVALID_ARG;
+    for (int i = 0; i < EOSQ_NUM_STAGES; ++i) {
+        ms[i] = 0.0f;
+        launches[i] = 0;
+    }
+    int rc = EOSQ_OK;
+    for (eosq_ctx::Timed &t : ctx->timed) {
+        float e = 0.0f;
+        if (record_cuda(ctx, cudaEventSynchronize(t.stop), "cudaEventSynchronize") ||
+            record_cuda(ctx, cudaEventElapsedTime(&e, t.start, t.stop), "cudaEventElapsedTime"))
+            rc = EOSQ_ERR_CUDA;
+        ms[t.stage] += e;
+        launches[t.stage] += 1;
+        ctx->free_events.push_back(t.start);
+        ctx->free_events.push_back(t.stop);
+    }
+    ctx->timed.clear();
+    return rc;
+}
+
+extern "C" const char *eosq_last_cuda_error(const eosq_ctx *ctx) { return ctx ? ctx->last_error.c_str() : ""; }
+
+extern "C" int64_t eosq_launch_count(const eosq_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+extern "C" int eosq_encode(eosq_ctx *ctx, const void *blocks, int in_dtype, int64_t num_blocks, int n, int d,
+                           int bits, uint64_t seed, const eosq_cache_t *out, void *workspace,
+                           size_t workspace_bytes, void *cuda_stream) {
+    if (!ctx || num_blocks < 0 || (in_dtype != EOSQ_F16 && in_dtype != EOSQ_F32)) return EOSQ_ERR_INVALID_ARG;
+    int rc = check_shape(n, d, bits);
+    if (rc != EOSQ_OK) return rc;
+    if (num_blocks == 0) return EOSQ_OK;
+    if (!blocks || !cache_required_ok(out) || !workspace) return EOSQ_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(blocks) & 15u) || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
+        (reinterpret_cast<uintptr_t>(out->codes) & 15u))
+        return EOSQ_ERR_INVALID_ARG;
+    if (workspace_bytes < eosq_workspace_bytes(num_blocks, n, d)) return EOSQ_ERR_BUFFER_TOO_SMALL;
+    Rotation rot;
+    Codebook cb;
+    if ((rc = get_rotation(ctx, d, seed, &rot)) != EOSQ_OK) return rc;
+    if ((rc = get_codebook(d, bits, &cb)) != EOSQ_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const int64_t cap = std::min<int64_t>(num_blocks, CHUNK_BLOCKS);
+    Workspace ws;
+    carve(workspace, cap, &ws);
+    const size_t esize = (in_dtype == EOSQ_F32) ? 4 : 2;
+    for (int64_t b0 = 0; b0 < num_blocks; b0 += cap) {
+        const int64_t nb = std::min<int64_t>(cap, num_blocks - b0);
+        const char *chunk_in = static_cast<const char *>(blocks) + static_cast<size_t>(b0) * n * D * esize;
+        const eosq_cache_t o = shifted(*out, b0, n, bits);
+        run_stage(ctx, ST_GRAM, s, [&] { launch_gram_plain(chunk_in, in_dtype, nb, n, ws.gram, s); });
+        run_stage(ctx, ST_TRIDIAG, s, [&] { launch_tridiag(nb, ws, nullptr, s); });
+        run_stage(ctx, ST_EIGVALS, s, [&] { launch_eigvals(nb, ws, s); });
+        run_stage(ctx, ST_SPECTRAL, s, [&] { launch_spectral(nb, n, ws, o, 0, s); });
+        run_stage(ctx, ST_QUANT, s, [&] { launch_quant_plain(chunk_in, in_dtype, nb, n, ws, rot, cb, o, 0, s); });
+    }
+    if (record_cuda(ctx, cudaGetLastError(), "eosq_encode launch")) return EOSQ_ERR_CUDA;
+    return EOSQ_OK;
+}
+
+extern "C" int eosq_decode(eosq_ctx *ctx, const eosq_cache_t *cache, int64_t num_blocks, int n, int d, int bits,
+                           uint64_t seed, void *out_blocks, int out_dtype, void *cuda_stream) {
+    if (!ctx || num_blocks < 0 || (out_dtype != EOSQ_F16 && out_dtype != EOSQ_F32)) return EOSQ_ERR_INVALID_ARG;
+    int rc = check_shape(n, d, bits);
+    if (rc != EOSQ_OK) return rc;
+    if (num_blocks == 0) return EOSQ_OK;
+    if (!cache || !cache->codes || !cache->norms || !cache->rank || !cache->P || !cache->V || !out_blocks)
+        return EOSQ_ERR_INVALID_ARG;
+    Rotation rot;
+    Codebook cb;
+    if ((rc = get_rotation(ctx, d, seed, &rot)) != EOSQ_OK) return rc;
+    if ((rc = get_codebook(d, bits, &cb)) != EOSQ_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    run_stage(ctx, ST_DECODE, s, [&] { launch_decode_plain(*cache, num_blocks, n, rot, cb, out_blocks, out_dtype, s); });
+    if (record_cuda(ctx, cudaGetLastError(), "eosq_decode launch")) return EOSQ_ERR_CUDA;
+    return EOSQ_OK;
+}
+
+extern "C" int eosq_scores(eosq_ctx *ctx, const eosq_cache_t *kcache, int64_t num_kv_heads, int64_t blocks_per_head,
+                           int64_t head_stride_blocks, int n, int d, int bits, uint64_t seed, const void *q, int G,
+                           float scale, float *scores, void *cuda_stream) {
+    if (!ctx || num_kv_heads < 0 || blocks_per_head < 0 || head_stride_blocks < blocks_per_head || G < 1)
+        return EOSQ_ERR_INVALID_ARG;
+    int rc = check_shape(n, d, bits);
+    if (rc != EOSQ_OK) return rc;
+    if (num_kv_heads == 0 || blocks_per_head == 0) return EOSQ_OK;
+    if (!kcache || !kcache->codes || !kcache->norms || !kcache->rank || !kcache->P || !kcache->V || !q || !scores)
+        return EOSQ_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(kcache->codes) & 3u) return EOSQ_ERR_INVALID_ARG;
+    Rotation rot;
+    Codebook cb;
+    if ((rc = get_rotation(ctx, d, seed, &rot)) != EOSQ_OK) return rc;
+    if ((rc = get_codebook(d, bits, &cb)) != EOSQ_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    run_stage(ctx, ST_SCORES, s, [&] {
+        launch_scores_plain(*kcache, num_kv_heads, blocks_per_head, head_stride_blocks, n, rot, cb,
+                            static_cast<const __half *>(q), G, scale, scores, s);
+    });
+    if (record_cuda(ctx, cudaGetLastError(), "eosq_scores launch")) return EOSQ_ERR_CUDA;
+    return EOSQ_OK;
+}
+
+// ---- host-buffer path ----------------------------------------------------------------------
+namespace {
+constexpr int64_t HOST_CHUNK = 1184;
+
+struct Arena {
+    void *in;
+    eosq_cache_t dev;
+    void *ws;
+    size_t ws_bytes;
+};
+
+size_t carve_arena(void *base, int64_t cap, int n, int bits, int in_dtype, Arena *a) {
+    char *p = static_cast<char *>(base);
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        void *q = p ? p + off : nullptr;
+        off = align_up(off + bytes, 256);
+        return q;
+    };
+    Arena r;
+    std::memset(&r, 0, sizeof(r));
+    const size_t esize = (in_dtype == EOSQ_F32) ? 4 : 2;
+    r.in = take(static_cast<size_t>(cap) * n * D * esize);
+    r.dev.codes = static_cast<uint8_t *>(take(static_cast<size_t>(cap) * n * D * bits / 8));
+    r.dev.norms = static_cast<uint16_t *>(take(static_cast<size_t>(cap) * n * 2));
+    r.dev.rank = static_cast<int32_t *>(take(static_cast<size_t>(cap) * 4));
+    r.dev.sigma = static_cast<float *>(take(static_cast<size_t>(cap) * RMAX * 4));
+    r.dev.phi = static_cast<float *>(take(static_cast<size_t>(cap) * RMAX * 4));
+    r.dev.P = static_cast<uint16_t *>(take(static_cast<size_t>(cap) * RMAX * n * 2));
+    r.dev.V = static_cast<uint16_t *>(take(static_cast<size_t>(cap) * RMAX * D * 2));
+    r.dev.status = static_cast<int32_t *>(take(static_cast<size_t>(cap) * 4));
+    r.dev.eig = static_cast<float *>(take(static_cast<size_t>(cap) * D * 4));
+    r.dev.lambda_plus = static_cast<float *>(take(static_cast<size_t>(cap) * 4));
+    r.ws_bytes = eosq_workspace_bytes(cap, n, D);
+    r.ws = take(r.ws_bytes);
+    if (a) *a = r;
+    return off;
+}
+}  // namespace
+
+extern "C" size_t eosq_encode_host_arena_bytes(int64_t num_blocks, int n, int d, int bits, int in_dtype) {
+    if (num_blocks <= 0 || check_shape(n, d, bits) != EOSQ_OK) return 0;
+    return carve_arena(nullptr, std::min<int64_t>(num_blocks, HOST_CHUNK), n, bits, in_dtype, nullptr);
+}
+
+extern "C" int eosq_encode_host(eosq_ctx *ctx, const void *host_blocks, int in_dtype, int64_t num_blocks, int n,
+                                int d, int bits, uint64_t seed, const eosq_cache_t *host_out, void *arena,
+                                size_t arena_bytes, void *cuda_stream) {
+    if (!ctx || num_blocks < 0 || (in_dtype != EOSQ_F16 && in_dtype != EOSQ_F32)) return EOSQ_ERR_INVALID_ARG;
+    int rc = check_shape(n, d, bits);
+    if (rc != EOSQ_OK) return rc;
+    if (num_blocks == 0) return EOSQ_OK;
+    if (!host_blocks || !cache_required_ok(host_out) || !arena || (reinterpret_cast<uintptr_t>(arena) & 255u))
+        return EOSQ_ERR_INVALID_ARG;
+    if (arena_bytes < eosq_encode_host_arena_bytes(num_blocks, n, d, bits, in_dtype)) return EOSQ_ERR_BUFFER_TOO_SMALL;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const int64_t cap = std::min<int64_t>(num_blocks, HOST_CHUNK);
+    Arena a;
+    carve_arena(arena, cap, n, bits, in_dtype, &a);
+    const size_t esize = (in_dtype == EOSQ_F32) ? 4 : 2;
+    const size_t rb = static_cast<size_t>(D) * bits / 8;
+    for (int64_t b0 = 0; b0 < num_blocks; b0 += cap) {
+        const int64_t nb = std::min<int64_t>(cap, num_blocks - b0);
+        const char *src = static_cast<const char *>(host_blocks) + static_cast<size_t>(b0) * n * D * esize;
+        if (record_cuda(ctx, cudaMemcpyAsync(a.in, src, static_cast<size_t>(nb) * n * D * esize, cudaMemcpyHostToDevice, s), "h2d"))
+            return EOSQ_ERR_CUDA;
+        eosq_cache_t dev = a.dev;
+        if (!host_out->eig) dev.eig = nullptr;
+        if (!host_out->lambda_plus) dev.lambda_plus = nullptr;
+        rc = eosq_encode(ctx, a.in, in_dtype, nb, n, d, bits, seed, &dev, a.ws, a.ws_bytes, s);
+        if (rc != EOSQ_OK) return rc;
+        const eosq_cache_t h = shifted(*host_out, b0, n, bits);
+        cudaError_t e = cudaSuccess;
+        auto back = [&](void *dst, const void *srcp, size_t bytes) {
+            if (e == cudaSuccess && dst) e = cudaMemcpyAsync(dst, srcp, bytes, cudaMemcpyDeviceToHost, s);
+        };
+        back(h.codes, dev.codes, static_cast<size_t>(nb) * n * rb);
+        back(h.norms, dev.norms, static_cast<size_t>(nb) * n * 2);
+        back(h.rank, dev.rank, static_cast<size_t>(nb) * 4);
+        back(h.sigma, dev.sigma, static_cast<size_t>(nb) * RMAX * 4);
+        back(h.phi, dev.phi, static_cast<size_t>(nb) * RMAX * 4);
+        back(h.P, dev.P, static_cast<size_t>(nb) * RMAX * n * 2);
+        back(h.V, dev.V, static_cast<size_t>(nb) * RMAX * D * 2);
+        back(h.status, dev.status, static_cast<size_t>(nb) * 4);
+        if (dev.eig) back(h.eig, dev.eig, static_cast<size_t>(nb) * D * 4);
+        if (dev.lambda_plus) back(h.lambda_plus, dev.lambda_plus, static_cast<size_t>(nb) * 4);
+        if (record_cuda(ctx, e, "d2h")) return EOSQ_ERR_CUDA;
+    }
+    if (record_cuda(ctx, cudaStreamSynchronize(s), "cudaStreamSynchronize")) return EOSQ_ERR_CUDA;
+    return EOSQ_OK;
+}
+
+extern "C" int eosq_check_status(eosq_ctx *ctx, const int32_t *status, int64_t num_blocks, int64_t *flagged,
+                                 void *cuda_stream) {
+    if (!ctx || num_blocks < 0 || (num_blocks > 0 && !status)) return EOSQ_ERR_INVALID_ARG;
+    std::vector<int32_t> h(static_cast<size_t>(num_blocks));
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    if (num_blocks > 0) {
+        if (record_cuda(ctx, cudaMemcpyAsync(h.data(), status, sizeof(int32_t) * h.size(), cudaMemcpyDeviceToHost, s), "status copy"))
+            return EOSQ_ERR_CUDA;
+    }
+    if (record_cuda(ctx, cudaStreamSynchronize(s), "cudaStreamSynchronize")) return EOSQ_ERR_CUDA;
+    int64_t cnt = 0;
+    for (int32_t v : h) cnt += (v != 0);
+    if (flagged) *flagged = cnt;
+    return cnt ? EOSQ_WARN_BLOCK_STATUS : EOSQ_OK;
+}

@@ -1,0 +1,109 @@
+// Shared declarations of the eosq CUDA library (sm_100a): constants, the context, the
+// workspace view and the kernel launchers implemented in the other translation units.
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+#include <string>
+#include <vector>
+
+#include "eosq.h"
+
+namespace eosq {
+
+constexpr int D = 128;         // head dimension the kernels are written for
+constexpr int RMAX = EOSQ_RMAX;
+constexpr int KPILOT = 11;     // floor(128^(1/2.01)), checked against eosq_pilot_k at create time
+constexpr int NMAX = 4096;
+
+// Lloyd-Max codebook as kernel parameter (fp32 copies of the host doubles).
+struct Codebook {
+    float centroid[16];
+    float threshold[15];
+    int bits;
+};
+
+// Device copies of one seeded rotation.
+struct Rotation {
+    uint64_t seed = 0;
+    float *pi = nullptr;     // [c][j]  z_c = sum_j pi[c][j] u_j
+    float *pi_t = nullptr;   // [j][c]
+};
+
+// Scratch of one chunk of blocks, carved out of the caller's workspace.
+struct Workspace {
+    double *gram;   // [C][D][D]   Gram matrix, later the Householder vectors (rows, right of the superdiagonal)
+    double *diag;   // [C][D]      tridiagonal diagonal
+    double *off;    // [C][D]      tridiagonal off-diagonal (D-1 used)
+    double *tau;    // [C][D]      Householder scalars (D-2 used)
+    double *lam;    // [C][D]      eigenvalues, descending
+    float *vr;      // [C][RMAX][D] right vectors as used for the residual
+    float *coef;    // [C][RMAX]   phi_i / sigma_i
+    int *rank;      // [C]
+};
+
+constexpr size_t WS_PER_BLOCK = sizeof(double) * (D * D + 4 * D) + sizeof(float) * (RMAX * D + RMAX) + 64;
+constexpr int64_t CHUNK_BLOCKS = 592;  // 4 per SM on 148 SMs: the scratch of one chunk stays L2 sized
+
+}  // namespace eosq
+
+enum Stage { ST_GRAM = 0, ST_TRIDIAG, ST_EIGVALS, ST_SPECTRAL, ST_QUANT, ST_DECODE, ST_SCORES, ST_OTHER };
+
+struct eosq_ctx {
+    struct Timed {
+        int stage;
+        cudaEvent_t start, stop;
+    };
+    int device = 0;
+    std::vector<eosq::Rotation> rotations;
+    std::string last_error;
+    int64_t launches = 0;
+    bool profile = false;
+    std::vector<Timed> timed;
+    std::vector<cudaEvent_t> free_events;
+};
+
+namespace eosq {
+
+// ---- launchers (each enqueues one kernel on `stream`) ---------------------------------------
+// Gram matrix G = S^T S of each block, accumulated in double from exact products.
+void launch_gram_plain(const void *blocks, int in_dtype, int64_t nb, int n, double *gram, cudaStream_t s);
+// Householder tridiagonalisation of each Gram matrix (in place: reflectors overwrite it).
+void launch_tridiag(int64_t nb, const Workspace &ws, int *status, cudaStream_t s);
+// All eigenvalues of each tridiagonal matrix by Sturm bisection.
+void launch_eigvals(int64_t nb, const Workspace &ws, cudaStream_t s);
+// Bulk edge, rank, imputed spectrum, D-transform and shrinkage; kept eigenvectors.
+void launch_spectral(int64_t nb, int n, const Workspace &ws, const eosq_cache_t &out, int64_t block0,
+                     cudaStream_t s);
+// Residual, norm, rotation, codes, packing and left factors.
+void launch_quant_plain(const void *blocks, int in_dtype, int64_t nb, int n, const Workspace &ws,
+                        const Rotation &rot, const Codebook &cb, const eosq_cache_t &out, int64_t block0,
+                        cudaStream_t s);
+void launch_decode_plain(const eosq_cache_t &cache, int64_t nb, int n, const Rotation &rot, const Codebook &cb,
+                         void *out_blocks, int out_dtype, cudaStream_t s);
+void launch_scores_plain(const eosq_cache_t &cache, int64_t heads, int64_t bph, int64_t head_stride, int n,
+                         const Rotation &rot, const Codebook &cb, const __half *q, int G, float scale,
+                         float *scores, cudaStream_t s);
+
+// ---- small device helpers -------------------------------------------------------------------
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+template <typename T>
+__device__ __forceinline__ float load_as_float(const T *p);
+template <>
+__device__ __forceinline__ float load_as_float<float>(const float *p) { return *p; }
+template <>
+__device__ __forceinline__ float load_as_float<__half>(const __half *p) { return __half2float(*p); }
+
+}  // namespace eosq

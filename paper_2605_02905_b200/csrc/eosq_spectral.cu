@@ -1,0 +1,445 @@
+// Spectral stage of eosq_encode: symmetric eigen-decomposition of the d x d Gram matrix
+// (the block's singular values and right singular vectors, Sec. 2.3) and Algorithm 2
+// (bulk edge, rank, imputed noise spectrum, D-transform estimators, Frobenius shrinker).
+//
+// All arithmetic here is double precision: the bulk eigenvalues sit two to three orders of
+// magnitude below the largest outlier, and the rank test and the shrunk values must agree with a
+// double-precision reference to 1e-4 relative or better.
+#include "eosq_common.cuh"
+
+namespace eosq {
+
+// ------------------------------------------------------------------------------------------
+// Householder tridiagonalisation, one CTA per matrix, matrix resident in shared memory.
+// Step k reflects row k right of the superdiagonal; the reflector (v[k+1] = 1 implied) is left
+// in row k, columns k+2.., for the back-transformation of eigenvectors.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) tridiag_kernel(double *__restrict__ gram, double *__restrict__ diag,
+                                                      double *__restrict__ off, double *__restrict__ tau) {
+    extern __shared__ double A[];  // D * D
+    __shared__ double v[D], p[D];
+    __shared__ double s_tau;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    double *G = gram + static_cast<size_t>(blockIdx.x) * D * D;
+    double *dg = diag + static_cast<size_t>(blockIdx.x) * D;
+    double *of = off + static_cast<size_t>(blockIdx.x) * D;
+    double *ta = tau + static_cast<size_t>(blockIdx.x) * D;
+    for (int e = tid; e < D * D; e += 256) A[e] = G[e];
+    __syncthreads();
+
+    for (int k = 0; k < D - 2; ++k) {
+        if (warp == 0) {
+            const double alpha = A[k * D + k + 1];
+            double ss = 0.0;
+            for (int j = k + 2 + lane; j < D; j += 32) {
+                const double x = A[k * D + j];
+                ss += x * x;
+            }
+            ss = warp_sum(ss);
+            double beta = alpha, t = 0.0, scale = 0.0;
+            if (ss > 0.0) {
+                beta = -copysign(sqrt(alpha * alpha + ss), alpha);
+                t = (beta - alpha) / beta;
+                scale = 1.0 / (alpha - beta);
+            }
+            for (int j = k + 2 + lane; j < D; j += 32) {
+                const double x = A[k * D + j] * scale;
+                v[j] = x;
+                A[k * D + j] = x;
+            }
+            if (lane == 0) {
+                v[k + 1] = 1.0;
+                s_tau = t;
+                dg[k] = A[k * D + k];
+                of[k] = beta;
+                ta[k] = t;
+            }
+        }
+        __syncthreads();
+        const double t = s_tau;
+        if (t != 0.0) {
+            // p = t * A22 v   (one warp per row of the trailing matrix)
+            for (int i = k + 1 + warp; i < D; i += 8) {
+                double acc = 0.0;
+                for (int j = k + 1 + lane; j < D; j += 32) acc += A[i * D + j] * v[j];
+                acc = warp_sum(acc);
+                if (lane == 0) p[i] = t * acc;
+            }
+            __syncthreads();
+            // w = p - (t/2)(p.v) v ;  A22 -= v w^T + w v^T
+            double dot = 0.0;
+            for (int j = k + 1 + lane; j < D; j += 32) dot += p[j] * v[j];
+            dot = warp_sum(dot);
+            const double kk = -0.5 * t * dot;
+            for (int i = k + 1 + warp; i < D; i += 8) {
+                const double vi = v[i], wi = p[i] + kk * vi;
+                for (int j = k + 1 + lane; j < D; j += 32) {
+                    const double vj = v[j], wj = p[j] + kk * vj;
+                    A[i * D + j] -= vi * wj + wi * vj;
+                }
+            }
+        }
+        __syncthreads();
+    }
+    if (tid == 0) {
+        dg[D - 2] = A[(D - 2) * D + D - 2];
+        of[D - 2] = A[(D - 2) * D + D - 1];
+        dg[D - 1] = A[(D - 1) * D + D - 1];
+        of[D - 1] = 0.0;
+        ta[D - 2] = 0.0;
+        ta[D - 1] = 0.0;
+    }
+    for (int e = tid; e < D * D; e += 256) G[e] = A[e];
+}
+
+// ------------------------------------------------------------------------------------------
+// Eigenvalues of a symmetric tridiagonal matrix by bisection on the Sturm sequence
+//   p_0 = 1, p_1 = d_0 - x, p_{i+1} = (d_i - x) p_i - e_{i-1}^2 p_{i-1};
+// the number of sign changes is the number of eigenvalues below x.  One thread per eigenvalue.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ int sturm_count(const double *sd, const double *se2, double x) {
+    double p0 = 1.0, p1 = sd[0] - x;
+    bool neg = !(p1 > 0.0);  // an exact zero takes the sign opposite to its predecessor
+    int cnt = neg ? 1 : 0;
+#pragma unroll 4
+    for (int i = 1; i < D; ++i) {
+        const double p2 = (sd[i] - x) * p1 - se2[i - 1] * p0;
+        const bool neg2 = (p2 < 0.0) || (p2 == 0.0 && !neg);
+        cnt += (neg2 != neg) ? 1 : 0;
+        neg = neg2;
+        p0 = p1;
+        p1 = p2;
+        const double m = fmax(fabs(p0), fabs(p1));
+        if (!(m > 1e-100 && m < 1e100)) {
+            if (m > 0.0 && m < 1e308) {
+                const double r = 1.0 / m;
+                p0 *= r;
+                p1 *= r;
+            } else {  // both vanished (decoupled block hit exactly): restart with the current sign
+                p0 = 0.0;
+                p1 = neg ? -1.0 : 1.0;
+            }
+        }
+    }
+    return cnt;
+}
+
+constexpr int BISECT_ITERS = 50;
+
+__global__ void __launch_bounds__(D) eigvals_kernel(const double *__restrict__ diag, const double *__restrict__ off,
+                                                    double *__restrict__ lam) {
+    __shared__ double sd[D], se2[D];
+    __shared__ double s_red[4];
+    const int tid = threadIdx.x;
+    const size_t base = static_cast<size_t>(blockIdx.x) * D;
+    const double d0 = diag[base + tid];
+    const double e0 = (tid < D - 1) ? off[base + tid] : 0.0;
+    double m = fmax(fabs(d0), fabs(e0));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmax(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if ((tid & 31) == 0) s_red[tid >> 5] = m;
+    __syncthreads();
+    m = fmax(fmax(s_red[0], s_red[1]), fmax(s_red[2], s_red[3]));
+    const double scale = (m > 0.0 && m < 1e300) ? 1.0 / m : 1.0;
+    sd[tid] = d0 * scale;
+    se2[tid] = (e0 * scale) * (e0 * scale);
+    __syncthreads();
+    const int target = D - 1 - tid;  // ascending index of the eigenvalue this thread brackets
+    double lo = -3.0, hi = 3.0;      // Gershgorin bound once every entry is at most 1 in magnitude
+    for (int it = 0; it < BISECT_ITERS; ++it) {
+        const double mid = 0.5 * (lo + hi);
+        if (sturm_count(sd, se2, mid) > target) hi = mid;
+        else lo = mid;
+    }
+    lam[base + tid] = 0.5 * (lo + hi) / scale;
+}
+
+// ------------------------------------------------------------------------------------------
+// Algorithm 2 on the spectrum, then the kept eigenvectors by inverse iteration on the
+// tridiagonal matrix and back-transformation through the stored reflectors.
+// ------------------------------------------------------------------------------------------
+constexpr int LU_LANES = 16;
+constexpr size_t SPECTRAL_DYN_SMEM = sizeof(double) * (4 * D * LU_LANES + LU_LANES * D);
+
+__global__ void __launch_bounds__(256) spectral_kernel(int n, Workspace ws, eosq_cache_t out, long long block0) {
+    __shared__ double lam[D], dd[D], ee[D], tt[D], atoms[D];
+    __shared__ double s_phi[RMAX], s_sig[RMAX];
+    __shared__ unsigned s_flags;
+    extern __shared__ double dyn[];
+    double *lu_l = dyn;                      // multipliers            [D][16]
+    double *lu_d = dyn + D * LU_LANES;       // reciprocal pivots      [D][16]
+    double *lu_u = dyn + 2 * D * LU_LANES;   // first superdiagonal    [D][16]
+    double *lu_u2 = dyn + 3 * D * LU_LANES;  // second superdiagonal   [D][16]
+    double *yv = dyn + 4 * D * LU_LANES;     // iteration vectors      [D][16]
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int b = blockIdx.x;
+    const long long gb = block0 + b;
+    const size_t base = static_cast<size_t>(b) * D;
+    if (tid < D) {
+        lam[tid] = ws.lam[base + tid];
+        dd[tid] = ws.diag[base + tid];
+        ee[tid] = ws.off[base + tid];
+        tt[tid] = ws.tau[base + tid];
+    }
+    if (tid < RMAX) {
+        s_phi[tid] = 0.0;
+        s_sig[tid] = 0.0;
+    }
+    if (tid == 0) s_flags = 0u;
+    __syncthreads();
+
+    // Step 1: bulk edge from lambda_{k+1}, lambda_{2k+1} (1-based) and the rank test.
+    const double edge_c = 1.0 / (cbrt(4.0) - 1.0);
+    const double cut = 1.0 / cbrt(static_cast<double>(D));
+    const double lam_plus = lam[KPILOT] + edge_c * (lam[KPILOT] - lam[2 * KPILOT]);
+    const bool pass = (tid < D) && (lam[tid] / lam_plus - 1.0 > cut);
+    int rank = __syncthreads_count(pass);
+    if (tid == 0) {
+        unsigned f = 0u;
+        if (!(lam[0] == lam[0]) || !(lam[0] < 1e300) || !(lam_plus == lam_plus)) f |= EOSQ_BLOCK_NONFINITE;
+        if (rank > KPILOT) f |= EOSQ_BLOCK_NONFINITE;
+        if (f) atomicOr(&s_flags, f);
+    }
+    if (rank > KPILOT) rank = KPILOT;
+
+    if (rank > 0) {
+        // Step 2: k imputed atoms behind the outliers, observed eigenvalues after them.
+        if (tid < D) {
+            double a = 0.0;
+            if (tid >= rank + KPILOT) a = lam[tid];
+            else if (tid >= rank) {
+                const int jj = tid - rank + 1;
+                const double bs = lam[KPILOT + rank];
+                const double gap = bs - lam[2 * KPILOT + rank];
+                a = bs + (1.0 - pow(static_cast<double>(jj) / KPILOT, 2.0 / 3.0)) * edge_c * gap;
+            }
+            atoms[tid] = a;
+        }
+        __syncthreads();
+        // Step 3: Stieltjes transforms of F_e at z = lambda_i, D-transform, Eq. 9, Eq. 6.
+        for (int i = warp; i < rank; i += 8) {
+            const double z = lam[i];
+            double ms = 0.0, msp = 0.0;
+            for (int j = rank + lane; j < D; j += 32) {
+                const double inv = 1.0 / (atoms[j] - z);
+                ms += inv;
+                msp += inv * inv;
+            }
+            ms = warp_sum(ms);
+            msp = warp_sum(msp);
+            if (lane == 0) {
+                const double nn = static_cast<double>(D - rank);
+                ms /= nn;
+                msp /= nn;
+                const double ratio = static_cast<double>(D) / static_cast<double>(n);
+                const double m1 = ratio * ms - (1.0 - ratio) / z;  // n x n side: n - d extra zeros
+                const double m1p = ratio * msp + (1.0 - ratio) / (z * z);
+                const double m2 = ms, m2p = msp;                   // d x d side
+                const double T = z * m1 * m2;
+                const double Tp = m1 * m2 + z * (m1p * m2 + m1 * m2p);
+                const double dh = 1.0 / sqrt(T);
+                const double a1 = m1 / (dh * dh * Tp), a2 = m2 / (dh * dh * Tp);
+                double ph = dh * sqrt(a1 * a2);
+                const double sg = sqrt(z);
+                if (!(ph >= 0.0) || !(ph < 1e300)) {
+                    ph = 0.0;
+                    atomicOr(&s_flags, EOSQ_BLOCK_CLAMPED);
+                } else if (ph > sg) {
+                    ph = sg;
+                    atomicOr(&s_flags, EOSQ_BLOCK_CLAMPED);
+                }
+                s_phi[i] = ph;
+                s_sig[i] = sg;
+                if (i > 0 && (lam[i - 1] - z) < 1e-9 * lam[i - 1]) atomicOr(&s_flags, EOSQ_BLOCK_CLUSTERED);
+            }
+        }
+
+        // Kept eigenvectors of the tridiagonal matrix: (T - mu I) = P L U with partial pivoting,
+        // three steps of inverse iteration.  Lane i of warp 0 owns vector i (column i of the arrays).
+        if (warp == 0 && lane < rank) {
+            const int c = lane;
+            const double mu = lam[c];
+            const double floor_piv = 1.2e-16 * fmax(fabs(lam[0]), 1e-300);
+            unsigned piv[4] = {0u, 0u, 0u, 0u};
+            double d_i = dd[0] - mu, u_i = ee[0];
+            for (int i = 0; i < D - 1; ++i) {
+                const double l = ee[i];
+                const double d_next = dd[i + 1] - mu;
+                const double u_next = (i + 1 < D - 1) ? ee[i + 1] : 0.0;
+                double fact, nd, nu;
+                if (fabs(d_i) >= fabs(l)) {
+                    fact = (d_i != 0.0) ? l / d_i : 0.0;
+                    lu_d[i * LU_LANES + c] = d_i;
+                    lu_u[i * LU_LANES + c] = u_i;
+                    lu_u2[i * LU_LANES + c] = 0.0;
+                    nd = d_next - fact * u_i;
+                    nu = u_next;
+                } else {
+                    fact = d_i / l;
+                    lu_d[i * LU_LANES + c] = l;
+                    lu_u[i * LU_LANES + c] = d_next;
+                    lu_u2[i * LU_LANES + c] = u_next;
+                    nd = u_i - fact * d_next;
+                    nu = -fact * u_next;
+                    piv[i >> 5] |= 1u << (i & 31);
+                }
+                lu_l[i * LU_LANES + c] = fact;
+                d_i = nd;
+                u_i = nu;
+            }
+            lu_d[(D - 1) * LU_LANES + c] = d_i;
+            lu_u[(D - 1) * LU_LANES + c] = 0.0;
+            lu_u2[(D - 1) * LU_LANES + c] = 0.0;
+            for (int i = 0; i < D; ++i) {
+                double x = lu_d[i * LU_LANES + c];
+                if (!(fabs(x) >= floor_piv)) x = (x < 0.0) ? -floor_piv : floor_piv;
+                lu_d[i * LU_LANES + c] = 1.0 / x;
+            }
+            for (int i = 0; i < D; ++i) {
+                const double f = (i + 1) * 0.6180339887498949;
+                yv[i * LU_LANES + c] = 0.5 + (f - floor(f));
+            }
+            for (int it = 0; it < 3; ++it) {
+                double carry = yv[c];
+                for (int i = 0; i < D - 1; ++i) {  // forward: apply the row interchanges and L^-1
+                    const double next = yv[(i + 1) * LU_LANES + c];
+                    const double l = lu_l[i * LU_LANES + c];
+                    if ((piv[i >> 5] >> (i & 31)) & 1u) {
+                        yv[i * LU_LANES + c] = next;
+                        carry = carry - l * next;
+                    } else {
+                        yv[i * LU_LANES + c] = carry;
+                        carry = next - l * carry;
+                    }
+                }
+                double x1 = carry * lu_d[(D - 1) * LU_LANES + c];  // backward: U^-1
+                yv[(D - 1) * LU_LANES + c] = x1;
+                double x2 = 0.0, ss = x1 * x1;
+                for (int i = D - 2; i >= 0; --i) {
+                    const double x = (yv[i * LU_LANES + c] - lu_u[i * LU_LANES + c] * x1 - lu_u2[i * LU_LANES + c] * x2) *
+                                     lu_d[i * LU_LANES + c];
+                    yv[i * LU_LANES + c] = x;
+                    ss += x * x;
+                    x2 = x1;
+                    x1 = x;
+                }
+                // normalise in two steps so that the squares cannot overflow
+                const double big = sqrt(ss);
+                const double inv = (big > 0.0 && big < 1e300) ? 1.0 / big : 1.0;
+                if (!(big > 0.0 && big < 1e300)) atomicOr(&s_flags, EOSQ_BLOCK_NOT_CONVERGED);
+                for (int i = 0; i < D; ++i) yv[i * LU_LANES + c] *= inv;
+            }
+        }
+    }
+    __syncthreads();
+
+    // Back-transformation x = H_0 H_1 ... H_{D-3} y, one warp per pair of vectors (i, i + 8).
+    const double *R = ws.gram + static_cast<size_t>(b) * D * D;
+    float *vr = ws.vr + static_cast<size_t>(b) * RMAX * D;
+    if (warp < rank) {
+        const int i0 = warp, i1 = warp + 8;
+        const bool two = i1 < rank;
+        double y0[4], y1[4];
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+            y0[m] = yv[(lane + 32 * m) * LU_LANES + i0];
+            y1[m] = two ? yv[(lane + 32 * m) * LU_LANES + i1] : 0.0;
+        }
+        for (int k = D - 3; k >= 0; --k) {
+            const double t = tt[k];
+            if (t == 0.0) continue;
+            const double *row = R + static_cast<size_t>(k) * D;
+            double vv[4], dot0 = 0.0, dot1 = 0.0;
+#pragma unroll
+            for (int m = 0; m < 4; ++m) {
+                const int j = lane + 32 * m;
+                vv[m] = (j > k + 1) ? row[j] : ((j == k + 1) ? 1.0 : 0.0);
+                dot0 += vv[m] * y0[m];
+                dot1 += vv[m] * y1[m];
+            }
+            dot0 = t * warp_sum(dot0);
+            dot1 = t * warp_sum(dot1);
+#pragma unroll
+            for (int m = 0; m < 4; ++m) {
+                y0[m] -= dot0 * vv[m];
+                y1[m] -= dot1 * vv[m];
+            }
+        }
+        double n0 = 0.0, n1 = 0.0;
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+            n0 += y0[m] * y0[m];
+            n1 += y1[m] * y1[m];
+        }
+        n0 = warp_sum(n0);
+        n1 = warp_sum(n1);
+        const double r0 = (n0 > 0.0) ? rsqrt(n0) : 0.0, r1 = (n1 > 0.0) ? rsqrt(n1) : 0.0;
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+            const int j = lane + 32 * m;
+            const float f0 = static_cast<float>(y0[m] * r0);
+            vr[i0 * D + j] = f0;
+            out.V[(gb * RMAX + i0) * D + j] = __half_as_ushort(__float2half_rn(f0));
+            if (out.vr32) out.vr32[(gb * RMAX + i0) * D + j] = f0;
+            if (two) {
+                const float f1 = static_cast<float>(y1[m] * r1);
+                vr[i1 * D + j] = f1;
+                out.V[(gb * RMAX + i1) * D + j] = __half_as_ushort(__float2half_rn(f1));
+                if (out.vr32) out.vr32[(gb * RMAX + i1) * D + j] = f1;
+            }
+        }
+    }
+    // rows >= rank of V are zero; scalars
+    for (int e = tid; e < RMAX * D; e += 256) {
+        if (e / D >= rank) {
+            out.V[gb * RMAX * D + e] = 0;
+            vr[e] = 0.0f;
+            if (out.vr32) out.vr32[gb * RMAX * D + e] = 0.0f;
+        }
+    }
+    if (tid < RMAX) {
+        const float sg = static_cast<float>(s_sig[tid]);
+        const float ph = static_cast<float>(s_phi[tid]);
+        const float cf = (tid < rank && s_sig[tid] > 0.0) ? static_cast<float>(s_phi[tid] / s_sig[tid]) : 0.0f;
+        out.sigma[gb * RMAX + tid] = sg;
+        out.phi[gb * RMAX + tid] = ph;
+        ws.coef[static_cast<size_t>(b) * RMAX + tid] = cf;
+        if (out.coef) out.coef[gb * RMAX + tid] = cf;
+    }
+    if (tid < D && out.eig) out.eig[gb * D + tid] = static_cast<float>(lam[tid]);
+    if (tid == 0) {
+        out.rank[gb] = rank;
+        ws.rank[b] = rank;
+        out.status[gb] = static_cast<int32_t>(s_flags);
+        if (out.lambda_plus) out.lambda_plus[gb] = static_cast<float>(lam_plus);
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+void launch_tridiag(int64_t nb, const Workspace &ws, int *, cudaStream_t s) {
+    static bool configured = false;
+    const size_t smem = sizeof(double) * D * D;
+    if (!configured) {
+        cudaFuncSetAttribute(tridiag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+        configured = true;
+    }
+    tridiag_kernel<<<static_cast<unsigned>(nb), 256, smem, s>>>(ws.gram, ws.diag, ws.off, ws.tau);
+}
+
+void launch_eigvals(int64_t nb, const Workspace &ws, cudaStream_t s) {
+    eigvals_kernel<<<static_cast<unsigned>(nb), D, 0, s>>>(ws.diag, ws.off, ws.lam);
+}
+
+void launch_spectral(int64_t nb, int n, const Workspace &ws, const eosq_cache_t &out, int64_t block0,
+                     cudaStream_t s) {
+    static bool configured = false;
+    if (!configured) {
+        cudaFuncSetAttribute(spectral_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(SPECTRAL_DYN_SMEM));
+        configured = true;
+    }
+    spectral_kernel<<<static_cast<unsigned>(nb), 256, SPECTRAL_DYN_SMEM, s>>>(n, ws, out, static_cast<long long>(block0));
+}
+
+}  // namespace eosq

@@ -1,0 +1,240 @@
+"""GPU parity tests: the CUDA library, called through its C ABI, against the CPU oracle on the
+same seeded blocks.  Sizes span several tiles and ragged tails; the full-size case is checked on
+sampled blocks in the launch configuration the benchmark times."""
+import ctypes
+import json
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2605_02905_b200 as eosq
+from paper_2605_02905_b200 import synth
+
+import parity
+
+pytestmark = pytest.mark.gpu
+
+SEED = 1234
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    from paper_2605_02905_b200 import build
+    build.build()
+    c = eosq.Context()
+    yield c
+    c.close()
+
+
+def _encode(ctx, blocks_cpu, bits, seed=SEED):
+    dev = blocks_cpu.cuda()
+    cache = eosq.eosq_encode(ctx, dev, bits, seed)
+    torch.cuda.synchronize()
+    return dev, cache
+
+
+def _report(name, rep):
+    print(f"\n[parity] {name}: " + json.dumps({k: (round(v, 9) if isinstance(v, float) else v) for k, v in rep.items()}))
+
+
+def test_pr1_reference_block(ctx):
+    """Config 0: one 256 x 128 fp32 block, b = 2, rotation seed 0; three spikes kept, the fourth rejected."""
+    w = synth.pr1_block(0)
+    dev, cache = _encode(ctx, w.blocks, 2, seed=0)
+    rep, enc = parity.compare_encode(w.blocks, cache, 2, 0)
+    _report("pr1", rep)
+    assert int(cache.rank[0]) == 3 and rep["rank_mismatch"] == 0
+    assert rep["e2e_mismatch_out_band"] == 0
+    dec = eosq.eosq_decode(ctx, cache, 0)
+    parity.compare_decode(cache, dec, 2, 0)
+
+
+@pytest.mark.parametrize("bits", [1, 2, 3, 4])
+def test_small_fp16_blocks_all_bit_widths(ctx, bits):
+    w = synth.kv_cache_blocks("small", layers=1, kv_heads=2, tokens=768, n=256, rank_hi=8, seed=20 + bits)
+    dev, cache = _encode(ctx, w.blocks, bits)
+    rep, enc = parity.compare_encode(w.blocks, cache, bits, SEED)
+    _report(f"small_b{bits}", rep)
+    assert rep["e2e_out_band_fraction"] < 1e-4
+    for out_dtype in (torch.float32, torch.float16):
+        dec = eosq.eosq_decode(ctx, cache, SEED, out_dtype=out_dtype)
+        parity.compare_decode(cache, dec, bits, SEED, tol=1e-4 if out_dtype == torch.float32 else 1e-3)
+
+
+def test_llama_shaped_blocks_n1024(ctx):
+    """Config 1 prefix: keys and values of the first heads, n = 1024, spikes, coloured noise, outlier channels."""
+    w = synth.llama_1layer(max_blocks=20)
+    pick = [0, 1, 7, 8, 9, 15, 16, 19]  # K blocks 0..7, V blocks 8..15, next head's K 16..
+    dev, cache = _encode(ctx, w.blocks, 2)
+    rep, enc = parity.compare_encode(w.blocks, cache, 2, SEED, blocks_idx=pick)
+    _report("llama_n1024", rep)
+    assert rep["e2e_out_band_fraction"] < 1e-4
+    dec = eosq.eosq_decode(ctx, cache, SEED)
+    parity.compare_decode(cache, dec, 2, SEED, blocks_idx=pick[:4])
+
+
+def test_scores_match_oracle(ctx):
+    """Keys-only view of a [head][K|V][block] cache: G = 4 query heads per KV head, and a wide group."""
+    w = synth.kv_cache_blocks("scores", layers=1, kv_heads=3, tokens=512, n=256, rank_hi=6, seed=31)
+    heads, bph = 3, 2
+    for bits, G in ((2, 4), (3, 4), (4, 11), (1, 1)):
+        dev, cache = _encode(ctx, w.blocks, bits)
+        q = synth.queries(heads, G, seed=5).cuda()
+        scale = 1.0 / math.sqrt(128)
+        s = eosq.eosq_scores(ctx, cache, q, heads, bph, 2 * bph, SEED, scale)
+        torch.cuda.synchronize()
+        worst = parity.compare_scores(cache, q, s, heads, bph, 2 * bph, bits, SEED, scale)
+        print(f"\n[parity] scores b={bits} G={G}: worst relative {worst:.3e}")
+
+
+def test_degenerate_blocks(ctx):
+    """Pure noise (rank 0), an all-zero block, a block with zero rows, a rank-one block."""
+    g = torch.Generator().manual_seed(3)
+    n, d = 256, 128
+    noise = torch.randn(n, d, generator=g) * 0.3
+    zero = torch.zeros(n, d)
+    holes = torch.randn(n, d, generator=g) * 0.3
+    holes[5] = 0
+    holes[200:210] = 0
+    rank1 = torch.randn(n, 1, generator=g) @ torch.randn(1, d, generator=g) + 0.05 * torch.randn(n, d, generator=g)
+    blocks = torch.stack([noise, zero, holes, rank1]).to(torch.float16)
+    dev, cache = _encode(ctx, blocks, 2)
+    rep, enc = parity.compare_encode(blocks, cache, 2, SEED)
+    _report("degenerate", rep)
+    ranks = cache.rank.cpu().tolist()
+    assert ranks[0] == 0 and ranks[1] == 0 and ranks[2] == 0 and ranks[3] == 1
+    norms = cache.norms.cpu()
+    assert torch.all(norms[1] == 0) and norms[2][5] == 0 and torch.all(norms[2][200:210] == 0)
+    dec = eosq.eosq_decode(ctx, cache, SEED)
+    assert torch.all(dec[1] == 0) and torch.all(dec[2][5] == 0)
+    parity.compare_decode(cache, dec, 2, SEED)
+
+
+@pytest.mark.parametrize("n", [128, 136, 4096])
+def test_ragged_and_extreme_block_lengths(ctx, n):
+    """n = d (square), n not a multiple of the row tile, and the largest supported n."""
+    w = synth.kv_cache_blocks("ragged", layers=1, kv_heads=1, tokens=2 * n, n=n, rank_hi=5, seed=40 + n)
+    dev, cache = _encode(ctx, w.blocks, 3)
+    rep, enc = parity.compare_encode(w.blocks, cache, 3, SEED, blocks_idx=[0, 3] if n == 4096 else None)
+    _report(f"n{n}", rep)
+    dec = eosq.eosq_decode(ctx, cache, SEED)
+    parity.compare_decode(cache, dec, 3, SEED, blocks_idx=[0] if n == 4096 else None)
+    q = synth.queries(2, 4, seed=6).cuda()
+    s = eosq.eosq_scores(ctx, cache, q, 2, 2, 2, SEED)
+    parity.compare_scores(cache, q, s, 2, 2, 2, 3, SEED, 1.0 / math.sqrt(128), pairs=[(0, 0), (1, 1)])
+
+
+def test_many_blocks_cross_the_chunk_boundary_and_are_deterministic(ctx):
+    """More blocks than one internal chunk: every block must equal its stand-alone encoding."""
+    w = synth.kv_cache_blocks("chunks", layers=2, kv_heads=3, tokens=128 * 51, n=128, rank_hi=4, seed=50)
+    assert w.blocks.shape[0] == 612
+    dev, cache = _encode(ctx, w.blocks, 2)
+    dev2, cache2 = _encode(ctx, w.blocks, 2)
+    for name in ("codes", "norms", "rank", "sigma", "phi", "V", "status", "eig"):
+        assert torch.equal(getattr(cache, name), getattr(cache2, name)), name
+    pick = [0, 591, 592, 611]
+    for b in pick:
+        _, single = _encode(ctx, w.blocks[b:b + 1], 2)
+        assert torch.equal(single.codes[0], cache.codes[b]) and torch.equal(single.norms[0], cache.norms[b])
+        r = int(single.rank[0])
+        assert r == int(cache.rank[b]) and torch.equal(single.P[0, :r], cache.P[b, :r])
+    rep, enc = parity.compare_encode(w.blocks, cache, 2, SEED, blocks_idx=pick)
+    _report("chunks", rep)
+
+
+def test_host_buffer_entry_point_matches_device_path(ctx):
+    w = synth.kv_cache_blocks("host", layers=1, kv_heads=2, tokens=512, n=256, rank_hi=6, seed=60)
+    dev, cache = _encode(ctx, w.blocks, 2)
+    B, n, d = w.blocks.shape
+    host_in = w.blocks.pin_memory()
+    host_out = eosq.Cache.allocate(B, n, d, 2, pinned=True, diagnostics=False)
+    host_out.eig = torch.empty((B, d), dtype=torch.float32).pin_memory()
+    arena = torch.empty(eosq.eosq_encode_host_arena_bytes(B, n, d, 2, eosq.EOSQ_F16), dtype=torch.uint8, device="cuda")
+    eosq.eosq_encode_host(ctx, host_in, 2, SEED, host_out, arena)
+    for name in ("codes", "norms", "rank", "sigma", "phi", "V", "status", "eig"):
+        assert torch.equal(getattr(host_out, name), getattr(cache, name).cpu()), name
+    for b in range(B):
+        r = int(cache.rank[b])
+        assert torch.equal(host_out.P[b, :r], cache.P[b, :r].cpu())
+
+
+def test_empty_input_and_argument_errors(ctx):
+    L = eosq.lib()
+    empty = torch.empty((0, 256, 128), dtype=torch.float16, device="cuda")
+    cache = eosq.eosq_encode(ctx, empty, 2, SEED)
+    assert cache.num_blocks == 0
+    assert eosq.eosq_decode(ctx, cache, SEED).shape == (0, 256, 128)
+    blocks = torch.zeros((2, 256, 128), dtype=torch.float16, device="cuda")
+    good = eosq.Cache.allocate(2, 256, 128, 2)
+    st = good.struct()
+    ws = torch.empty(eosq.eosq_workspace_bytes(2, 256, 128), dtype=torch.uint8, device="cuda")
+    stream = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+    def call(blocks_ptr=blocks.data_ptr(), dtype=eosq.EOSQ_F16, B=2, n=256, d=128, bits=2, out=ctypes.addressof(st),
+             wsp=ws.data_ptr(), wsb=ws.numel()):
+        return L.eosq_encode(ctx._h, blocks_ptr, dtype, B, n, d, bits, ctypes.c_uint64(SEED), out, wsp, wsb, stream)
+
+    assert call() == eosq.EOSQ_OK
+    assert call(blocks_ptr=None) == eosq.EOSQ_ERR_INVALID_ARG
+    assert call(out=None) == eosq.EOSQ_ERR_INVALID_ARG
+    assert call(dtype=7) == eosq.EOSQ_ERR_INVALID_ARG
+    assert call(B=-1) == eosq.EOSQ_ERR_INVALID_ARG
+    assert call(blocks_ptr=blocks.data_ptr() + 2) == eosq.EOSQ_ERR_INVALID_ARG
+    assert call(d=64) == eosq.EOSQ_ERR_UNSUPPORTED
+    assert call(bits=5) == eosq.EOSQ_ERR_UNSUPPORTED
+    assert call(n=64) == eosq.EOSQ_ERR_UNSUPPORTED
+    assert call(n=8192) == eosq.EOSQ_ERR_UNSUPPORTED
+    assert call(wsb=1024) == eosq.EOSQ_ERR_BUFFER_TOO_SMALL
+    missing = eosq.Cache.allocate(2, 256, 128, 2)
+    missing.norms = None
+    st2 = missing.struct()
+    assert call(out=ctypes.addressof(st2)) == eosq.EOSQ_ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    assert eosq.eosq_check_status(ctx, good) == 0
+
+
+def test_nonfinite_input_is_flagged_not_fatal(ctx):
+    blocks = torch.randn(2, 256, 128, generator=torch.Generator().manual_seed(1)).to(torch.float16)
+    blocks[1, 3, 7] = float("inf")
+    dev, cache = _encode(ctx, blocks, 2)
+    status = cache.status.cpu().tolist()
+    assert status[0] == 0 and status[1] != 0
+    assert eosq.eosq_check_status(ctx, cache) == 1
+
+
+def test_full_size_cache_sampled_blocks(ctx):
+    """Config 2 in the benchmark's launch configuration: the whole Llama-3.1-8B-shaped 32k cache
+    (16384 blocks, 4 GiB) is encoded in one call; sampled blocks go to the oracle one by one, and
+    properties that hold at any size are checked on everything."""
+    w = synth.llama_32k(device="cuda")
+    B = w.blocks.shape[0]
+    assert B == 16384
+    cache = eosq.eosq_encode(ctx, w.blocks, 2, SEED)
+    torch.cuda.synchronize()
+    assert eosq.eosq_check_status(ctx, cache) == 0
+    ranks = cache.rank
+    assert int(ranks.min()) >= 0 and int(ranks.max()) <= 11
+    eig = cache.eig
+    assert torch.all(eig[:, :-1] >= eig[:, 1:]) and torch.all(eig[:, -1] > -1e-3 * eig[:, 0])
+    assert torch.all(torch.isfinite(cache.norms.float()))
+    # Frobenius identity: sum of eigenvalues of the Gram matrix = ||S||_F^2
+    fro = (w.blocks[:256].float() ** 2).sum(dim=(1, 2))
+    assert torch.allclose(eig[:256].sum(dim=1), fro, rtol=2e-3)
+    pick = [0, 31, 32, 4097, 9000, B - 1]
+    sub = w.blocks[pick].cpu()
+    sub_cache = eosq.Cache.allocate(len(pick), w.n, w.d, 2)
+    for name in ("codes", "norms", "rank", "sigma", "phi", "P", "V", "status", "eig", "lambda_plus", "vr32", "coef"):
+        getattr(sub_cache, name).copy_(getattr(cache, name)[pick])
+    rep, enc = parity.compare_encode(sub, sub_cache, 2, SEED)
+    _report("llama_32k_sampled", rep)
+    assert rep["e2e_out_band_fraction"] < 1e-4
+    # scores over the keys of the first layers, sampled (head, block) pairs against the oracle
+    heads, bph, G = 16, 32, 4
+    q = synth.queries(heads, G, seed=8).cuda()
+    s = eosq.eosq_scores(ctx, cache, q, heads, bph, 2 * bph, SEED)
+    torch.cuda.synchronize()
+    parity.compare_scores(cache, q, s, heads, bph, 2 * bph, 2, SEED, 1.0 / math.sqrt(128), pairs=[(0, 0), (5, 17), (15, 31)])
