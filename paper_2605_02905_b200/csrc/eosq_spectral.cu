@@ -140,7 +140,13 @@ __global__ void __launch_bounds__(D) eigvals_kernel(const double *__restrict__ d
     if ((tid & 31) == 0) s_red[tid >> 5] = m;
     __syncthreads();
     m = fmax(fmax(s_red[0], s_red[1]), fmax(s_red[2], s_red[3]));
-    const double scale = (m > 0.0 && m < 1e300) ? 1.0 / m : 1.0;
+    // a non-finite entry anywhere poisons the whole spectrum: report NaN instead of a bracket
+    const int bad = __syncthreads_or(!(fabs(d0) < 1e300) || !(fabs(e0) < 1e300));
+    if (bad) {
+        lam[base + tid] = nan("");
+        return;
+    }
+    const double scale = (m > 0.0) ? 1.0 / m : 1.0;
     sd[tid] = d0 * scale;
     se2[tid] = (e0 * scale) * (e0 * scale);
     __syncthreads();

@@ -79,9 +79,12 @@ class Workload:
 
 
 def _orthonormal(gen, batch, rows, cols, device):
-    g = torch.randn(batch, rows, cols, generator=gen, device=device, dtype=torch.float32)
-    q, _ = torch.linalg.qr(g)
-    return q
+    """Orthonormal columns from a Gaussian draw, by Cholesky-QR in double (two batched calls
+    instead of one factorisation per matrix): Q = G L^-T with G^T G = L L^T."""
+    g = torch.randn(batch, rows, cols, generator=gen, device=device, dtype=torch.float32).double()
+    chol = torch.linalg.cholesky(g.transpose(1, 2) @ g)
+    q = torch.linalg.solve_triangular(chol, g.transpose(1, 2), upper=False).transpose(1, 2)
+    return q.float()
 
 
 def spiked_blocks(num_blocks, n, d, *, ranks, theta_mult, sigma_col, alpha, outlier=None,
