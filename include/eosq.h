@@ -131,6 +131,35 @@ int eosq_encode(eosq_ctx *ctx, const void *blocks, int in_dtype, int64_t num_blo
                 size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * eosq_encode without any device allocation.  (The paper has no counterpart: this entry point
+ * exists for the sake of callers, not of the method.)
+ *
+ * Who needs it: code that must not call cudaMalloc where it compresses -- a serving loop whose
+ * device memory was divided up at start-up, a plug-in that was given buffers but no allocator, a
+ * caller that has begun capturing a stream.  eosq_encode makes such callers bring a workspace and
+ * allocates the device copy of the rotation on the first use of a seed; this variant does
+ * neither.  Its scratch and its copy of the rotation live in one fixed array in the library's
+ * device image (about 4.7 MB, held by every GPU that loads the library until the process exits).
+ * The call itself performs no cudaMalloc, no cudaFree and no allocating library call.
+ *
+ * Arguments and results are those of eosq_encode (same kernels, same outputs) minus the
+ * workspace.  Limits and rules:
+ *   - num_blocks <= EOSQ_STATIC_MAX_BLOCKS; a larger count is rejected with
+ *     EOSQ_ERR_BUFFER_TOO_SMALL (text in eosq_last_cuda_error) and nothing is enqueued.
+ *   - The first call on a device looks up the array's device address (that device must be
+ *     current, as for every call), and the first call with a new seed uploads that seed's
+ *     rotation from host memory on the given stream.  Make those calls before any stream capture.
+ *   - All calls on a device share the one array, and it keeps whatever the last call left.  The
+ *     kernels write every scratch value before reading it, so nothing needs clearing, but two
+ *     calls that overlap on the GPU (different streams, no ordering between them) race; order
+ *     them on one stream or with events.  Calls are serialised on the host by a lock.
+ */
+#define EOSQ_STATIC_MAX_BLOCKS 32
+int64_t eosq_encode_static_max_blocks(void);
+int eosq_encode_static(eosq_ctx *ctx, const void *blocks, int in_dtype, int64_t num_blocks, int n, int d,
+                       int bits, uint64_t seed, const eosq_cache_t *out, void *cuda_stream);
+
+/*
  * Reconstruct blocks from a compressed cache (Algorithm 1 last TQ_MSE line, Algorithm 2 Return):
  *   x_hat[t] = sum_{i<r} P[i][t] V[i][:] + norms[t] * Pi^T centroids[codes[t]].
  *   out_blocks dev [num_blocks][n][d] of out_dtype (EOSQ_F16 or EOSQ_F32).

@@ -27,6 +27,7 @@ EXPORTS = [
     "eosq_workspace_bytes", "eosq_create", "eosq_destroy", "eosq_last_cuda_error", "eosq_encode",
     "eosq_decode", "eosq_scores", "eosq_encode_host_arena_bytes", "eosq_encode_host",
     "eosq_check_status", "eosq_launch_count", "eosq_profile_enable", "eosq_profile_read",
+    "eosq_encode_static", "eosq_encode_static_max_blocks",
 ]
 STAGES = ["gram", "tridiag", "eigvals", "spectral", "quant", "decode", "scores", "other"]
 
@@ -78,6 +79,10 @@ def lib():
         L.eosq_destroy.argtypes = [ctypes.c_void_p]
         L.eosq_encode.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
                                   ctypes.c_int, ctypes.c_uint64, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+        L.eosq_encode_static.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
+                                         ctypes.c_int, ctypes.c_uint64, ctypes.c_void_p, ctypes.c_void_p]
+        L.eosq_encode_static_max_blocks.restype = ctypes.c_int64
+        L.eosq_encode_static_max_blocks.argtypes = []
         L.eosq_decode.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                   ctypes.c_uint64, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p]
         L.eosq_scores.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_int,
@@ -258,6 +263,26 @@ def eosq_encode(ctx: Context, blocks, bits: int, seed: int, out: Optional[Cache]
                            ctypes.c_uint64(seed), ctypes.addressof(st), workspace.data_ptr(), workspace.numel(),
                            _stream_ptr(stream))
     _check(rc, "eosq_encode", ctx)
+    return out
+
+
+def eosq_encode_static_max_blocks() -> int:
+    return int(lib().eosq_encode_static_max_blocks())
+
+
+def eosq_encode_static(ctx: Context, blocks, bits: int, seed: int, out: Cache, stream=None) -> Cache:
+    """``eosq_encode`` for callers that may not allocate device memory: no workspace argument, the
+    library's fixed device array serves as scratch.  ``out`` must be allocated by the caller
+    beforehand; at most ``eosq_encode_static_max_blocks()`` blocks per call.  This wrapper itself
+    creates no tensor."""
+    assert blocks.is_cuda and blocks.is_contiguous() and blocks.dim() == 3
+    B, n, d = blocks.shape
+    st = out.struct()
+    rc = lib().eosq_encode_static(ctx._h, blocks.data_ptr() if B else None, _dtype_code(blocks), B, n, d, bits,
+                                  ctypes.c_uint64(seed), ctypes.addressof(st), _stream_ptr(stream))
+    if rc == EOSQ_ERR_BUFFER_TOO_SMALL:
+        raise EosqError(rc, "eosq_encode_static", lib().eosq_last_cuda_error(ctx._h).decode())
+    _check(rc, "eosq_encode_static", ctx)
     return out
 
 

@@ -21,30 +21,6 @@ int check_shape(int n, int d, int bits) {
     return EOSQ_OK;
 }
 
-inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
-
-// Carve the scratch arrays of one chunk (capacity `cap` blocks) out of `base`.
-size_t carve(void *base, int64_t cap, Workspace *ws) {
-    char *p = static_cast<char *>(base);
-    size_t off = 0;
-    auto take = [&](size_t bytes) {
-        void *q = p ? p + off : nullptr;
-        off = align_up(off + bytes, 256);
-        return q;
-    };
-    Workspace w;
-    w.gram = static_cast<double *>(take(sizeof(double) * cap * D * D));
-    w.diag = static_cast<double *>(take(sizeof(double) * cap * D));
-    w.off = static_cast<double *>(take(sizeof(double) * cap * D));
-    w.tau = static_cast<double *>(take(sizeof(double) * cap * D));
-    w.lam = static_cast<double *>(take(sizeof(double) * cap * D));
-    w.vr = static_cast<float *>(take(sizeof(float) * cap * RMAX * D));
-    w.coef = static_cast<float *>(take(sizeof(float) * cap * RMAX));
-    w.rank = static_cast<int *>(take(sizeof(int) * cap));
-    if (ws) *ws = w;
-    return off;
-}
-
 int get_rotation(eosq_ctx *ctx, int d, uint64_t seed, Rotation *out) {
     for (const Rotation &r : ctx->rotations)
         if (r.seed == seed) {

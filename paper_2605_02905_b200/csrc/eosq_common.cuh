@@ -47,6 +47,31 @@ struct Workspace {
 constexpr size_t WS_PER_BLOCK = sizeof(double) * (D * D + 4 * D) + sizeof(float) * (RMAX * D + RMAX) + 64;
 constexpr int64_t CHUNK_BLOCKS = 592;  // 4 per SM on 148 SMs: the scratch of one chunk stays L2 sized
 
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Carve the scratch arrays of one chunk (capacity `cap` blocks) out of `base`; returns the bytes
+// used.  With base = nullptr only the size is computed.
+inline size_t carve(void *base, int64_t cap, Workspace *ws) {
+    char *p = static_cast<char *>(base);
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        void *q = p ? p + off : nullptr;
+        off = align_up(off + bytes, 256);
+        return q;
+    };
+    Workspace w;
+    w.gram = static_cast<double *>(take(sizeof(double) * cap * D * D));
+    w.diag = static_cast<double *>(take(sizeof(double) * cap * D));
+    w.off = static_cast<double *>(take(sizeof(double) * cap * D));
+    w.tau = static_cast<double *>(take(sizeof(double) * cap * D));
+    w.lam = static_cast<double *>(take(sizeof(double) * cap * D));
+    w.vr = static_cast<float *>(take(sizeof(float) * cap * RMAX * D));
+    w.coef = static_cast<float *>(take(sizeof(float) * cap * RMAX));
+    w.rank = static_cast<int *>(take(sizeof(int) * cap));
+    if (ws) *ws = w;
+    return off;
+}
+
 }  // namespace eosq
 
 enum Stage { ST_GRAM = 0, ST_TRIDIAG, ST_EIGVALS, ST_SPECTRAL, ST_QUANT, ST_DECODE, ST_SCORES, ST_OTHER };
