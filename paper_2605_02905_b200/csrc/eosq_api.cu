@@ -111,6 +111,39 @@ bool cache_required_ok(const eosq_cache_t *c) {
 
 }  // namespace
 
+// The launch sequence of eosq_encode for blocks [b0, b0 + nb) of `blocks`, with the scratch of
+// one chunk in `ws`.
+int eosq::encode_chunk(eosq_ctx *ctx, const void *blocks, int in_dtype, int64_t b0, int64_t nb, int n, int bits,
+                       const Rotation &rot, const Codebook &cb, const eosq_cache_t &out_all, const Workspace &ws,
+                       cudaStream_t s) {
+    const size_t esize = (in_dtype == EOSQ_F32) ? 4 : 2;
+    const char *chunk_in = static_cast<const char *>(blocks) + static_cast<size_t>(b0) * n * D * esize;
+    const eosq_cache_t o = shifted(out_all, b0, n, bits);
+    if (in_dtype == EOSQ_F16) {
+        bool setup_ok = true;
+        run_stage(ctx, ST_GRAM, s, [&] { setup_ok = launch_gram_tc(blocks, 0, b0, nb, n, ws.gram, ctx->dev_err, ctx->sm_count, s); });
+        if (!setup_ok) {
+            ctx->last_error = "tensor-core Gram kernel: tensor map or launch set-up failed";
+            return EOSQ_ERR_CUDA;
+        }
+    } else {
+        run_stage(ctx, ST_GRAM, s, [&] { launch_gram_plain(chunk_in, in_dtype, nb, n, ws.gram, nullptr, nullptr, s); });
+    }
+    run_stage(ctx, ST_TRIDIAG, s, [&] { launch_tridiag(nb, ws, nullptr, nullptr, s); });
+    run_stage(ctx, ST_EIGVALS, s, [&] { launch_eigvals(nb, ws, nullptr, nullptr, s); });
+    if (in_dtype == EOSQ_F16) {
+        // second pass, exact Gram matrix, for the blocks the tensor-core one cannot resolve
+        if (record_cuda(ctx, cudaMemsetAsync(ws.redo_count, 0, sizeof(int), s), "cudaMemsetAsync(redo count)")) return EOSQ_ERR_CUDA;
+        run_stage(ctx, ST_OTHER, s, [&] { launch_mark_redo(nb, ws, s); });
+        run_stage(ctx, ST_GRAM, s, [&] { launch_gram_plain(chunk_in, in_dtype, nb, n, ws.gram, ws.redo_list, ws.redo_count, s); });
+        run_stage(ctx, ST_TRIDIAG, s, [&] { launch_tridiag(nb, ws, ws.redo_list, ws.redo_count, s); });
+        run_stage(ctx, ST_EIGVALS, s, [&] { launch_eigvals(nb, ws, ws.redo_list, ws.redo_count, s); });
+    }
+    run_stage(ctx, ST_SPECTRAL, s, [&] { launch_spectral(nb, n, ws, o, 0, s); });
+    run_stage(ctx, ST_QUANT, s, [&] { launch_quant_plain(chunk_in, in_dtype, nb, n, ws, rot, cb, o, 0, s); });
+    return EOSQ_OK;
+}
+
 extern "C" size_t eosq_workspace_bytes(int64_t num_blocks, int n, int d) {
     (void)n;
     if (num_blocks <= 0 || d != D) return 0;
@@ -126,12 +159,20 @@ extern "C" int eosq_create(eosq_ctx **out) {
         delete ctx;
         return EOSQ_ERR_CUDA;
     }
+    cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device);
+    if (record_cuda(ctx, cudaMalloc(&ctx->dev_err, 256), "cudaMalloc(error word)") ||
+        record_cuda(ctx, cudaMemset(ctx->dev_err, 0, 256), "cudaMemset(error word)")) {
+        cudaFree(ctx->dev_err);
+        delete ctx;
+        return EOSQ_ERR_CUDA;
+    }
     *out = ctx;
     return EOSQ_OK;
 }
 
 extern "C" int eosq_destroy(eosq_ctx *ctx) {
     if (!ctx) return EOSQ_OK;
+    cudaFree(ctx->dev_err);
     for (Rotation &r : ctx->rotations) {
         cudaFree(r.pi);
         cudaFree(r.pi_t);
@@ -196,16 +237,10 @@ extern "C" int eosq_encode(eosq_ctx *ctx, const void *blocks, int in_dtype, int6
     const int64_t cap = std::min<int64_t>(num_blocks, CHUNK_BLOCKS);
     Workspace ws;
     carve(workspace, cap, &ws);
-    const size_t esize = (in_dtype == EOSQ_F32) ? 4 : 2;
     for (int64_t b0 = 0; b0 < num_blocks; b0 += cap) {
         const int64_t nb = std::min<int64_t>(cap, num_blocks - b0);
-        const char *chunk_in = static_cast<const char *>(blocks) + static_cast<size_t>(b0) * n * D * esize;
-        const eosq_cache_t o = shifted(*out, b0, n, bits);
-        run_stage(ctx, ST_GRAM, s, [&] { launch_gram_plain(chunk_in, in_dtype, nb, n, ws.gram, s); });
-        run_stage(ctx, ST_TRIDIAG, s, [&] { launch_tridiag(nb, ws, nullptr, s); });
-        run_stage(ctx, ST_EIGVALS, s, [&] { launch_eigvals(nb, ws, s); });
-        run_stage(ctx, ST_SPECTRAL, s, [&] { launch_spectral(nb, n, ws, o, 0, s); });
-        run_stage(ctx, ST_QUANT, s, [&] { launch_quant_plain(chunk_in, in_dtype, nb, n, ws, rot, cb, o, 0, s); });
+        rc = eosq::encode_chunk(ctx, blocks, in_dtype, b0, nb, n, bits, rot, cb, *out, ws, s);
+        if (rc != EOSQ_OK) return rc;
     }
     if (record_cuda(ctx, cudaGetLastError(), "eosq_encode launch")) return EOSQ_ERR_CUDA;
     return EOSQ_OK;
@@ -354,7 +389,14 @@ extern "C" int eosq_check_status(eosq_ctx *ctx, const int32_t *status, int64_t n
         if (record_cuda(ctx, cudaMemcpyAsync(h.data(), status, sizeof(int32_t) * h.size(), cudaMemcpyDeviceToHost, s), "status copy"))
             return EOSQ_ERR_CUDA;
     }
+    int dev_err = 0;
+    if (record_cuda(ctx, cudaMemcpyAsync(&dev_err, ctx->dev_err, sizeof(int), cudaMemcpyDeviceToHost, s), "error word copy"))
+        return EOSQ_ERR_CUDA;
     if (record_cuda(ctx, cudaStreamSynchronize(s), "cudaStreamSynchronize")) return EOSQ_ERR_CUDA;
+    if (dev_err != 0) {
+        ctx->last_error = "a bounded device-side wait gave up (kernel bits " + std::to_string(dev_err) + "); results are incomplete";
+        return EOSQ_ERR_CUDA;
+    }
     int64_t cnt = 0;
     for (int32_t v : h) cnt += (v != 0);
     if (flagged) *flagged = cnt;

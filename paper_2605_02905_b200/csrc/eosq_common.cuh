@@ -42,9 +42,16 @@ struct Workspace {
     float *vr;      // [C][RMAX][D] right vectors as used for the residual
     float *coef;    // [C][RMAX]   phi_i / sigma_i
     int *rank;      // [C]
+    int *redo_list; // [C]         blocks whose spectrum the tensor-core Gram matrix cannot resolve
+    int *redo_count;// [1]
 };
 
-constexpr size_t WS_PER_BLOCK = sizeof(double) * (D * D + 4 * D) + sizeof(float) * (RMAX * D + RMAX) + 64;
+constexpr size_t WS_PER_BLOCK = sizeof(double) * (D * D + 4 * D) + sizeof(float) * (RMAX * D + RMAX) + 64 + 8;
+// A block is redone with the exact (double precision) Gram matrix when its smallest eigenvalue is
+// below this fraction of its largest: the tensor-core Gram matrix carries an absolute error of
+// about 1e-8 of the largest eigenvalue, which would move smaller singular values by more than
+// 5e-5 relative.
+constexpr double REDO_RATIO = 1e-4;
 constexpr int64_t CHUNK_BLOCKS = 592;  // 4 per SM on 148 SMs: the scratch of one chunk stays L2 sized
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -68,6 +75,8 @@ inline size_t carve(void *base, int64_t cap, Workspace *ws) {
     w.vr = static_cast<float *>(take(sizeof(float) * cap * RMAX * D));
     w.coef = static_cast<float *>(take(sizeof(float) * cap * RMAX));
     w.rank = static_cast<int *>(take(sizeof(int) * cap));
+    w.redo_list = static_cast<int *>(take(sizeof(int) * cap));
+    w.redo_count = static_cast<int *>(take(sizeof(int)));
     if (ws) *ws = w;
     return off;
 }
@@ -82,6 +91,8 @@ struct eosq_ctx {
         cudaEvent_t start, stop;
     };
     int device = 0;
+    int sm_count = 148;
+    int *dev_err = nullptr;   // device word: bits raised by kernels whose bounded waits gave up
     std::vector<eosq::Rotation> rotations;
     std::string last_error;
     int64_t launches = 0;
@@ -92,13 +103,28 @@ struct eosq_ctx {
 
 namespace eosq {
 
+// The launch sequence of the encode path for blocks [b0, b0 + nb) of `blocks` (implemented with
+// the C entry points; shared by eosq_encode and eosq_encode_static).
+int encode_chunk(eosq_ctx *ctx, const void *blocks, int in_dtype, int64_t b0, int64_t nb, int n, int bits,
+                 const Rotation &rot, const Codebook &cb, const eosq_cache_t &out_all, const Workspace &ws,
+                 cudaStream_t s);
+
 // ---- launchers (each enqueues one kernel on `stream`) ---------------------------------------
 // Gram matrix G = S^T S of each block, accumulated in double from exact products.
-void launch_gram_plain(const void *blocks, int in_dtype, int64_t nb, int n, double *gram, cudaStream_t s);
+// With `list` given, CTA c works on block list[c] and CTAs c >= *count do nothing (same for the
+// two spectral launchers below).
+void launch_gram_plain(const void *blocks, int in_dtype, int64_t nb, int n, double *gram, const int *list,
+                       const int *count, cudaStream_t s);
+// Same result from the tensor cores (fp16 blocks only).  The chunk starts `block0` blocks into
+// `blocks_all`.  Returns false if the launch could not be set up (no kernel was enqueued).
+bool launch_gram_tc(const void *blocks_all, int64_t nb_all, int64_t block0, int64_t nb, int n, double *gram, int *err,
+                    int sm_count, cudaStream_t s);
 // Householder tridiagonalisation of each Gram matrix (in place: reflectors overwrite it).
-void launch_tridiag(int64_t nb, const Workspace &ws, int *status, cudaStream_t s);
+void launch_tridiag(int64_t nb, const Workspace &ws, const int *list, const int *count, cudaStream_t s);
 // All eigenvalues of each tridiagonal matrix by Sturm bisection.
-void launch_eigvals(int64_t nb, const Workspace &ws, cudaStream_t s);
+void launch_eigvals(int64_t nb, const Workspace &ws, const int *list, const int *count, cudaStream_t s);
+// Clears the redo list / appends every block whose eigenvalue range exceeds 1 / REDO_RATIO.
+void launch_mark_redo(int64_t nb, const Workspace &ws, cudaStream_t s);
 // Bulk edge, rank, imputed spectrum, D-transform and shrinkage; kept eigenvectors.
 void launch_spectral(int64_t nb, int n, const Workspace &ws, const eosq_cache_t &out, int64_t block0,
                      cudaStream_t s);

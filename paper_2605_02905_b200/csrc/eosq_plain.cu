@@ -15,10 +15,16 @@ constexpr int GRAM_ROWS = 32;
 
 template <typename Tin>
 __global__ void __launch_bounds__(256) gram_plain_kernel(const Tin *__restrict__ blocks, int n,
-                                                         double *__restrict__ gram) {
+                                                         double *__restrict__ gram, const int *__restrict__ list,
+                                                         const int *__restrict__ count) {
     __shared__ __align__(16) float tile[GRAM_ROWS][D];
     const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-    const Tin *S = blocks + static_cast<size_t>(blockIdx.x) * n * D;
+    int blk = blockIdx.x;
+    if (list) {
+        if (blk >= *count) return;
+        blk = list[blk];
+    }
+    const Tin *S = blocks + static_cast<size_t>(blk) * n * D;
     double acc[8][8];
 #pragma unroll
     for (int i = 0; i < 8; ++i)
@@ -44,7 +50,7 @@ __global__ void __launch_bounds__(256) gram_plain_kernel(const Tin *__restrict__
                 for (int j = 0; j < 8; ++j) acc[i][j] += a[i] * bb[j];
         }
     }
-    double *G = gram + static_cast<size_t>(blockIdx.x) * D * D;
+    double *G = gram + static_cast<size_t>(blk) * D * D;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         const int row = (i < 4) ? 4 * ty + i : 64 + 4 * ty + (i - 4);
@@ -56,11 +62,12 @@ __global__ void __launch_bounds__(256) gram_plain_kernel(const Tin *__restrict__
     }
 }
 
-void launch_gram_plain(const void *blocks, int in_dtype, int64_t nb, int n, double *gram, cudaStream_t s) {
+void launch_gram_plain(const void *blocks, int in_dtype, int64_t nb, int n, double *gram, const int *list,
+                       const int *count, cudaStream_t s) {
     if (in_dtype == EOSQ_F32)
-        gram_plain_kernel<float><<<static_cast<unsigned>(nb), 256, 0, s>>>(static_cast<const float *>(blocks), n, gram);
+        gram_plain_kernel<float><<<static_cast<unsigned>(nb), 256, 0, s>>>(static_cast<const float *>(blocks), n, gram, list, count);
     else
-        gram_plain_kernel<__half><<<static_cast<unsigned>(nb), 256, 0, s>>>(static_cast<const __half *>(blocks), n, gram);
+        gram_plain_kernel<__half><<<static_cast<unsigned>(nb), 256, 0, s>>>(static_cast<const __half *>(blocks), n, gram, list, count);
 }
 
 // ------------------------------------------------------------------------------------------

@@ -15,15 +15,21 @@ namespace eosq {
 // in row k, columns k+2.., for the back-transformation of eigenvectors.
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) tridiag_kernel(double *__restrict__ gram, double *__restrict__ diag,
-                                                      double *__restrict__ off, double *__restrict__ tau) {
+                                                      double *__restrict__ off, double *__restrict__ tau,
+                                                      const int *__restrict__ list, const int *__restrict__ count) {
     extern __shared__ double A[];  // D * D
     __shared__ double v[D], p[D];
     __shared__ double s_tau;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    double *G = gram + static_cast<size_t>(blockIdx.x) * D * D;
-    double *dg = diag + static_cast<size_t>(blockIdx.x) * D;
-    double *of = off + static_cast<size_t>(blockIdx.x) * D;
-    double *ta = tau + static_cast<size_t>(blockIdx.x) * D;
+    int blk = blockIdx.x;
+    if (list) {
+        if (blk >= *count) return;
+        blk = list[blk];
+    }
+    double *G = gram + static_cast<size_t>(blk) * D * D;
+    double *dg = diag + static_cast<size_t>(blk) * D;
+    double *of = off + static_cast<size_t>(blk) * D;
+    double *ta = tau + static_cast<size_t>(blk) * D;
     for (int e = tid; e < D * D; e += 256) A[e] = G[e];
     __syncthreads();
 
@@ -127,11 +133,17 @@ __device__ __forceinline__ int sturm_count(const double *sd, const double *se2, 
 constexpr int BISECT_ITERS = 50;
 
 __global__ void __launch_bounds__(D) eigvals_kernel(const double *__restrict__ diag, const double *__restrict__ off,
-                                                    double *__restrict__ lam) {
+                                                    double *__restrict__ lam, const int *__restrict__ list,
+                                                    const int *__restrict__ count) {
     __shared__ double sd[D], se2[D];
     __shared__ double s_red[4];
     const int tid = threadIdx.x;
-    const size_t base = static_cast<size_t>(blockIdx.x) * D;
+    int blk = blockIdx.x;
+    if (list) {
+        if (blk >= *count) return;
+        blk = list[blk];
+    }
+    const size_t base = static_cast<size_t>(blk) * D;
     const double d0 = diag[base + tid];
     const double e0 = (tid < D - 1) ? off[base + tid] : 0.0;
     double m = fmax(fabs(d0), fabs(e0));
@@ -423,18 +435,31 @@ __global__ void __launch_bounds__(256) spectral_kernel(int n, Workspace ws, eosq
 }
 
 // ------------------------------------------------------------------------------------------
-void launch_tridiag(int64_t nb, const Workspace &ws, int *, cudaStream_t s) {
+// Blocks whose smallest eigenvalue is not at least REDO_RATIO of the largest (this includes
+// non-finite spectra) are queued for a second pass with the exact Gram matrix.
+__global__ void mark_redo_kernel(const double *__restrict__ lam, int nb, int *__restrict__ list, int *__restrict__ count) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= nb) return;
+    const double hi = lam[static_cast<size_t>(b) * D], lo = lam[static_cast<size_t>(b) * D + D - 1];
+    if (!(lo >= REDO_RATIO * hi)) list[atomicAdd(count, 1)] = b;
+}
+
+void launch_mark_redo(int64_t nb, const Workspace &ws, cudaStream_t s) {
+    mark_redo_kernel<<<static_cast<unsigned>((nb + 255) / 256), 256, 0, s>>>(ws.lam, static_cast<int>(nb), ws.redo_list, ws.redo_count);
+}
+
+void launch_tridiag(int64_t nb, const Workspace &ws, const int *list, const int *count, cudaStream_t s) {
     static bool configured = false;
     const size_t smem = sizeof(double) * D * D;
     if (!configured) {
         cudaFuncSetAttribute(tridiag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
         configured = true;
     }
-    tridiag_kernel<<<static_cast<unsigned>(nb), 256, smem, s>>>(ws.gram, ws.diag, ws.off, ws.tau);
+    tridiag_kernel<<<static_cast<unsigned>(nb), 256, smem, s>>>(ws.gram, ws.diag, ws.off, ws.tau, list, count);
 }
 
-void launch_eigvals(int64_t nb, const Workspace &ws, cudaStream_t s) {
-    eigvals_kernel<<<static_cast<unsigned>(nb), D, 0, s>>>(ws.diag, ws.off, ws.lam);
+void launch_eigvals(int64_t nb, const Workspace &ws, const int *list, const int *count, cudaStream_t s) {
+    eigvals_kernel<<<static_cast<unsigned>(nb), D, 0, s>>>(ws.diag, ws.off, ws.lam, list, count);
 }
 
 void launch_spectral(int64_t nb, int n, const Workspace &ws, const eosq_cache_t &out, int64_t block0,

@@ -114,12 +114,8 @@ extern "C" int eosq_encode_static(eosq_ctx *ctx, const void *blocks, int in_dtyp
     // this call before it is read, so the previous call's contents are simply overwritten.
     Workspace ws;
     carve(pd.base + 2 * ROT_BYTES, num_blocks, &ws);
-    launch_gram_plain(blocks, in_dtype, num_blocks, n, ws.gram, s);
-    launch_tridiag(num_blocks, ws, nullptr, s);
-    launch_eigvals(num_blocks, ws, s);
-    launch_spectral(num_blocks, n, ws, *out, 0, s);
-    launch_quant_plain(blocks, in_dtype, num_blocks, n, ws, rot, cb, *out, 0, s);
-    ctx->launches += 5;
+    int rc = encode_chunk(ctx, blocks, in_dtype, 0, num_blocks, n, bits, rot, cb, *out, ws, s);
+    if (rc != EOSQ_OK) return rc;
     if (fail(ctx, cudaGetLastError(), "eosq_encode_static launch")) return EOSQ_ERR_CUDA;
     return EOSQ_OK;
 }
