@@ -140,7 +140,16 @@ int eosq::encode_chunk(eosq_ctx *ctx, const void *blocks, int in_dtype, int64_t 
         run_stage(ctx, ST_EIGVALS, s, [&] { launch_eigvals(nb, ws, ws.redo_list, ws.redo_count, s); });
     }
     run_stage(ctx, ST_SPECTRAL, s, [&] { launch_spectral(nb, n, ws, o, 0, s); });
-    run_stage(ctx, ST_QUANT, s, [&] { launch_quant_plain(chunk_in, in_dtype, nb, n, ws, rot, cb, o, 0, s); });
+    if (in_dtype == EOSQ_F16) {
+        bool setup_ok = true;
+        run_stage(ctx, ST_QUANT, s, [&] { setup_ok = launch_quant_tc(blocks, b0, nb, n, ws, rot, cb, o, ctx->dev_err, ctx->sm_count, s); });
+        if (!setup_ok) {
+            ctx->last_error = "tensor-core quantisation kernel: tensor map or launch set-up failed";
+            return EOSQ_ERR_CUDA;
+        }
+    } else {
+        run_stage(ctx, ST_QUANT, s, [&] { launch_quant_plain(chunk_in, in_dtype, nb, n, ws, rot, cb, o, 0, s); });
+    }
     return EOSQ_OK;
 }
 

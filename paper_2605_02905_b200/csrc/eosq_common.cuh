@@ -132,6 +132,9 @@ void launch_spectral(int64_t nb, int n, const Workspace &ws, const eosq_cache_t 
 void launch_quant_plain(const void *blocks, int in_dtype, int64_t nb, int n, const Workspace &ws,
                         const Rotation &rot, const Codebook &cb, const eosq_cache_t &out, int64_t block0,
                         cudaStream_t s);
+// Same outputs from the tensor cores (fp16 blocks only); `out` is already offset to the chunk.
+bool launch_quant_tc(const void *blocks_all, int64_t block0, int64_t nb, int n, const Workspace &ws, const Rotation &rot,
+                     const Codebook &cb, const eosq_cache_t &out, int *err, int sm_count, cudaStream_t s);
 void launch_decode_plain(const eosq_cache_t &cache, int64_t nb, int n, const Rotation &rot, const Codebook &cb,
                          void *out_blocks, int out_dtype, cudaStream_t s);
 void launch_scores_plain(const eosq_cache_t &cache, int64_t heads, int64_t bph, int64_t head_stride, int n,
