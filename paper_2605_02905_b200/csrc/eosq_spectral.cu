@@ -226,44 +226,58 @@ __global__ void __launch_bounds__(TD_THREADS, 1) tridiag_kernel(double *__restri
 }
 
 // ------------------------------------------------------------------------------------------
-// Eigenvalues of a symmetric tridiagonal matrix by bisection on the Sturm sequence
-//   p_0 = 1, p_1 = d_0 - x, p_{i+1} = (d_i - x) p_i - e_{i-1}^2 p_{i-1};
-// the number of sign changes is the number of eigenvalues below x.  One thread per eigenvalue.
+// Eigenvalues of a symmetric tridiagonal matrix from Sturm counts: with
+//   p_0 = 1, p_1 = d_0 - x, p_{i+1} = (d_i - x) p_i - e_{i-1}^2 p_{i-1},
+// the number of sign changes in p_0 .. p_d is the number of eigenvalues below x.  One thread per
+// eigenvalue.  A first pass counts at 128 points spaced geometrically below the Gershgorin bound
+// (the spectrum of a Gram matrix spans many decades), which brackets every eigenvalue to 18 %;
+// bisection then runs until the bracket is below 1e-10 relative (2e-15 of the matrix scale for the
+// smallest ones).
 // ------------------------------------------------------------------------------------------
-__device__ __forceinline__ int sturm_count(const double *sd, const double *se2, double x) {
-    double p0 = 1.0, p1 = sd[0] - x;
-    bool neg = !(p1 > 0.0);  // an exact zero takes the sign opposite to its predecessor
-    int cnt = neg ? 1 : 0;
-#pragma unroll 4
-    for (int i = 1; i < D; ++i) {
-        const double p2 = (sd[i] - x) * p1 - se2[i - 1] * p0;
-        const bool neg2 = (p2 < 0.0) || (p2 == 0.0 && !neg);
-        cnt += (neg2 != neg) ? 1 : 0;
-        neg = neg2;
-        p0 = p1;
-        p1 = p2;
-        const double m = fmax(fabs(p0), fabs(p1));
-        if (!(m > 1e-100 && m < 1e100)) {
-            if (m > 0.0 && m < 1e308) {
-                const double r = 1.0 / m;
-                p0 *= r;
-                p1 *= r;
-            } else {  // both vanished (decoupled block hit exactly): restart with the current sign
+constexpr double EV_E2_FLOOR = 1e-60;   // keeps the recurrence alive across an exactly decoupled entry
+constexpr int EV_MAX_BISECT = 64;
+
+// (d_i, e_{i-1}^2) pairs, scaled so that every entry is at most 1 in magnitude.
+__device__ __forceinline__ int sturm_count(const double2 *__restrict__ sde, double x) {
+    double p0 = 1.0, p1 = sde[0].x - x;
+    unsigned cnt = static_cast<unsigned>(__double2hiint(p1)) >> 31;
+#pragma unroll 1
+    for (int i0 = 1; i0 < D; i0 += 4) {
+#pragma unroll
+        for (int i = i0; i < i0 + 4; ++i) {
+            if (i < D) {
+                const double2 de = sde[i];
+                const double t = de.y * p0;
+                const double p2 = fma(de.x - x, p1, -t);
+                cnt += static_cast<unsigned>(__double2hiint(p1) ^ __double2hiint(p2)) >> 31;
+                p0 = p1;
+                p1 = p2;
+            }
+        }
+        // keep the pair within 2^+-300 of one
+        const int e0 = (__double2hiint(p0) >> 20) & 0x7ff, e1 = (__double2hiint(p1) >> 20) & 0x7ff;
+        const int em = max(e0, e1);
+        if (static_cast<unsigned>(em - 723) > 600u) {
+            if (em == 0) {   // both vanished: restart with the current sign
                 p0 = 0.0;
-                p1 = neg ? -1.0 : 1.0;
+                p1 = (__double2hiint(p1) < 0) ? -1.0 : 1.0;
+            } else if (em < 2047) {
+                const double sc = __hiloint2double((2046 - em) << 20, 0);
+                p0 *= sc;
+                p1 *= sc;
             }
         }
     }
-    return cnt;
+    return static_cast<int>(cnt);
 }
-
-constexpr int BISECT_ITERS = 50;
 
 __global__ void __launch_bounds__(D) eigvals_kernel(const double *__restrict__ diag, const double *__restrict__ off,
                                                     double *__restrict__ lam, const int *__restrict__ list,
                                                     const int *__restrict__ count) {
-    __shared__ double sd[D], se2[D];
-    __shared__ double s_red[4];
+    __shared__ __align__(16) double2 sde[D];
+    __shared__ double s_e2[D];
+    __shared__ double s_red[3][4];
+    __shared__ int s_cnt[D];
     const int tid = threadIdx.x;
     int blk = blockIdx.x;
     if (list) {
@@ -276,27 +290,65 @@ __global__ void __launch_bounds__(D) eigvals_kernel(const double *__restrict__ d
     double m = fmax(fabs(d0), fabs(e0));
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m = fmax(m, __shfl_xor_sync(0xffffffffu, m, o));
-    if ((tid & 31) == 0) s_red[tid >> 5] = m;
-    __syncthreads();
-    m = fmax(fmax(s_red[0], s_red[1]), fmax(s_red[2], s_red[3]));
+    if ((tid & 31) == 0) s_red[0][tid >> 5] = m;
     // a non-finite entry anywhere poisons the whole spectrum: report NaN instead of a bracket
     const int bad = __syncthreads_or(!(fabs(d0) < 1e300) || !(fabs(e0) < 1e300));
     if (bad) {
         lam[base + tid] = nan("");
         return;
     }
-    const double scale = (m > 0.0) ? 1.0 / m : 1.0;
-    sd[tid] = d0 * scale;
-    se2[tid] = (e0 * scale) * (e0 * scale);
+    m = fmax(fmax(s_red[0][0], s_red[0][1]), fmax(s_red[0][2], s_red[0][3]));
+    if (m == 0.0) {
+        lam[base + tid] = 0.0;
+        return;
+    }
+    const double scale = 1.0 / m;
+    const double sd = d0 * scale, se = fabs(e0 * scale);
+    s_e2[tid] = (tid < D - 1) ? fmax(se * se, EV_E2_FLOOR) : 0.0;
+    __syncthreads();
+    const double se_prev = (tid > 0) ? fabs(off[base + tid - 1] * scale) : 0.0;
+    sde[tid] = make_double2(sd, (tid > 0) ? s_e2[tid - 1] : 0.0);
+    // Gershgorin bounds of the scaled matrix
+    double glo = sd - se - se_prev, ghi = sd + se + se_prev;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        glo = fmin(glo, __shfl_xor_sync(0xffffffffu, glo, o));
+        ghi = fmax(ghi, __shfl_xor_sync(0xffffffffu, ghi, o));
+    }
+    if ((tid & 31) == 0) {
+        s_red[1][tid >> 5] = glo;
+        s_red[2][tid >> 5] = ghi;
+    }
+    __syncthreads();
+    glo = fmin(fmin(s_red[1][0], s_red[1][1]), fmin(s_red[1][2], s_red[1][3]));
+    ghi = fmax(fmax(s_red[2][0], s_red[2][1]), fmax(s_red[2][2], s_red[2][3]));
+    glo -= 1e-10 * (fabs(glo) + 1.0);
+    ghi += 1e-10 * (fabs(ghi) + 1.0);
+
+    // first pass: counts at D points, geometric below ghi when ghi > 0 (nine decades), else uniform
+    const bool geometric = ghi > 0.0;
+    auto point = [&](int t) -> double {
+        if (t < 0) return glo;
+        if (geometric) return ghi * exp2(-(9.0 * 3.321928094887362 / (D - 1)) * static_cast<double>(D - 1 - t));
+        return glo + (ghi - glo) * static_cast<double>(t + 1) / static_cast<double>(D);
+    };
+    s_cnt[tid] = sturm_count(sde, point(tid));
     __syncthreads();
     const int target = D - 1 - tid;  // ascending index of the eigenvalue this thread brackets
-    double lo = -3.0, hi = 3.0;      // Gershgorin bound once every entry is at most 1 in magnitude
-    for (int it = 0; it < BISECT_ITERS; ++it) {
+    int t = -1;                      // largest grid index with count <= target
+#pragma unroll
+    for (int step = D / 2; step > 0; step >>= 1)
+        if (t + step < D && s_cnt[t + step] <= target) t += step;
+    double lo = point(t), hi = (t + 1 < D) ? point(t + 1) : ghi;
+    if (t == D - 1) lo = hi;   // cannot happen (every eigenvalue is below the last point); keeps the bracket sane
+    for (int it = 0; it < EV_MAX_BISECT; ++it) {
         const double mid = 0.5 * (lo + hi);
-        if (sturm_count(sd, se2, mid) > target) hi = mid;
+        const bool done = (hi - lo) <= fmax(2e-15, 1e-10 * fabs(mid));
+        if (__all_sync(0xffffffffu, done)) break;
+        if (sturm_count(sde, mid) > target) hi = mid;
         else lo = mid;
     }
-    lam[base + tid] = 0.5 * (lo + hi) / scale;
+    lam[base + tid] = 0.5 * (lo + hi) * m;
 }
 
 // ------------------------------------------------------------------------------------------
