@@ -29,16 +29,167 @@ constexpr int TD_PLEN = 16 * TD_PSTRIDE;
 
 __device__ __forceinline__ int td_pos(int j) { return (j & 15) * TD_PSTRIDE + (j >> 4); }
 
+// Shared-memory state of one tridiagonalisation.
+struct TdShared {
+    double up[2][TD_PLEN];     // u, permuted (16-byte aligned by the struct's placement)
+    double pp[2][TD_PLEN];     // p, permuted
+    double wsum[2][8];
+    double sgam[2];
+    double dg[D], of[D], ta[D];
+};
+
+// The sixteen threads that hold row r (slot AR = r / 16 of their tiles) publish its tail as the
+// reflector of step r into buffer `nxt`.  Only slots b >= AR can hold columns j > r.
+template <int AR>
+__device__ __forceinline__ void td_publish(const double (&A)[8][8], int r, int nxt, int tc, int lane, TdShared &sh) {
+    const unsigned mask = 0xFFFFu << (lane & 16);
+    double x[8];
+    double ss0 = 0.0, ss1 = 0.0;
+#pragma unroll
+    for (int b = 0; b < 8; ++b) {
+        if (b < AR) {
+            x[b] = 0.0;
+        } else {
+            const int j = tc + 16 * b;
+            const double v = A[AR][b];
+            if (b == AR && j == r) sh.dg[r] = v;
+            x[b] = (j > r) ? v : 0.0;
+            const double t = (j > r + 1) ? v : 0.0;
+            if (b & 1) ss1 = fma(t, t, ss1);
+            else ss0 = fma(t, t, ss0);
+        }
+    }
+    double2 *dst = reinterpret_cast<double2 *>(&sh.up[nxt][tc * TD_PSTRIDE]);
+    dst[0] = make_double2(x[0], x[1]);
+    dst[1] = make_double2(x[2], x[3]);
+    dst[2] = make_double2(x[4], x[5]);
+    dst[3] = make_double2(x[6], x[7]);
+    double ss = ss0 + ss1;
+#pragma unroll
+    for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(mask, ss, o);
+    __syncwarp(mask);
+    const double alpha = sh.up[nxt][td_pos(r + 1)];
+    double beta = alpha, gamma = 0.0;
+    if (ss > 0.0) {
+        const double s2 = fma(alpha, alpha, ss);
+        const double nrm = s2 * rsqrt(s2);
+        beta = (alpha >= 0.0) ? -nrm : nrm;
+        gamma = 1.0 / fma(fabs(alpha), nrm, s2);   // 1 / (beta (beta - alpha))
+    }
+    __syncwarp(mask);
+    if (tc == 0) {
+        sh.up[nxt][td_pos(r + 1)] = alpha - beta;
+        sh.sgam[nxt] = gamma;
+        sh.of[r] = beta;
+        sh.ta[r] = gamma;
+    }
+}
+
+// One step k with (k + 1) / 16 == K0: tile slots below K0 hold only finished rows and columns and
+// are skipped at compile time.
+template <int K0>
+__device__ __forceinline__ void td_step(double (&A)[8][8], int k, int tid, TdShared &sh, double *__restrict__ refl) {
+    const int lane = tid & 31, warp = tid >> 5, tr = tid >> 4, tc = tid & 15;
+    __syncthreads();
+    const int cur = k & 1;
+    const double gamma = sh.sgam[cur];
+    if (tid < D) refl[k * D + tid] = (tid > k) ? sh.up[cur][td_pos(tid)] : 0.0;
+    const bool owner = (tr == ((k + 1) & 15)) && (k + 1 < D - 2);
+    if (gamma != 0.0) {   // uniform over the CTA
+        double uj[8], ui[8], acc[8];
+        {
+            const double2 *src = reinterpret_cast<const double2 *>(&sh.up[cur][tc * TD_PSTRIDE]);
+            const double2 *srow = reinterpret_cast<const double2 *>(&sh.up[cur][tr * TD_PSTRIDE]);
+#pragma unroll
+            for (int q = K0 / 2; q < 4; ++q) {
+                const double2 v = src[q], w = srow[q];
+                uj[2 * q] = v.x;
+                uj[2 * q + 1] = v.y;
+                ui[2 * q] = w.x;
+                ui[2 * q + 1] = w.y;
+            }
+        }
+        double tloc = 0.0;
+#pragma unroll
+        for (int a = 0; a < 8; ++a) {
+            acc[a] = 0.0;
+            if (a >= K0) {
+                double s0 = 0.0, s1 = 0.0;
+#pragma unroll
+                for (int b = K0; b < 8; ++b) {
+                    if ((b - K0) & 1) s1 = fma(A[a][b], uj[b], s1);
+                    else s0 = fma(A[a][b], uj[b], s0);
+                }
+                acc[a] = s0 + s1;
+                tloc = fma(ui[a], acc[a], tloc);
+            }
+        }
+        // sum the partial rows over the sixteen column groups: each stage keeps half of the rows
+        const bool h8 = tc & 8, h4 = tc & 4, h2 = tc & 2;
+        double v4[4], v2[2], v1;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const double keep = h8 ? acc[q + 4] : acc[q], send = h8 ? acc[q] : acc[q + 4];
+            v4[q] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+        }
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            const double keep = h4 ? v4[q + 2] : v4[q], send = h4 ? v4[q] : v4[q + 2];
+            v2[q] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+        }
+        {
+            const double keep = h2 ? v2[1] : v2[0], send = h2 ? v2[0] : v2[1];
+            v1 = keep + __shfl_xor_sync(0xffffffffu, send, 2);
+        }
+        v1 += __shfl_xor_sync(0xffffffffu, v1, 1);
+        const int arow = (h8 ? 4 : 0) + (h4 ? 2 : 0) + (h2 ? 1 : 0);
+        const int irow = tr + 16 * arow;
+        if (!(tc & 1) && irow > k) sh.pp[cur][td_pos(irow)] = gamma * v1;
+        tloc = warp_sum(tloc);
+        if (lane == 0) sh.wsum[cur][warp] = tloc;
+        __syncthreads();
+        const double2 w0 = *reinterpret_cast<const double2 *>(&sh.wsum[cur][0]), w1 = *reinterpret_cast<const double2 *>(&sh.wsum[cur][2]);
+        const double2 w2 = *reinterpret_cast<const double2 *>(&sh.wsum[cur][4]), w3 = *reinterpret_cast<const double2 *>(&sh.wsum[cur][6]);
+        const double uAu = ((w0.x + w0.y) + (w1.x + w1.y)) + ((w2.x + w2.y) + (w3.x + w3.y));
+        const double twoK = gamma * gamma * uAu;
+        double pj[8], si[8];
+        {
+            const double2 *src = reinterpret_cast<const double2 *>(&sh.pp[cur][tc * TD_PSTRIDE]);
+            const double2 *srow = reinterpret_cast<const double2 *>(&sh.pp[cur][tr * TD_PSTRIDE]);
+#pragma unroll
+            for (int q = K0 / 2; q < 4; ++q) {
+                const double2 v = src[q], w = srow[q];
+                pj[2 * q] = v.x;
+                pj[2 * q + 1] = v.y;
+                si[2 * q] = fma(-twoK, ui[2 * q], w.x);       // p_i - 2 K u_i
+                si[2 * q + 1] = fma(-twoK, ui[2 * q + 1], w.y);
+            }
+        }
+        // The next reflector comes from row k + 1 (slot K0 of its holders): bring that row up to
+        // date and publish it first, so that the other warps' updates hide its latency.
+        if (owner) {
+#pragma unroll
+            for (int b = K0; b < 8; ++b) A[K0][b] = fma(-ui[K0], pj[b], fma(-si[K0], uj[b], A[K0][b]));
+            td_publish<K0>(A, k + 1, cur ^ 1, tc, lane, sh);
+        }
+#pragma unroll
+        for (int a = K0; a < 8; ++a) {
+            if (a > K0 || !owner) {
+#pragma unroll
+                for (int b = K0; b < 8; ++b) A[a][b] = fma(-ui[a], pj[b], fma(-si[a], uj[b], A[a][b]));
+            }
+        }
+    } else if (owner) {
+        td_publish<K0>(A, k + 1, cur ^ 1, tc, lane, sh);
+    }
+}
+
 __global__ void __launch_bounds__(TD_THREADS, 1) tridiag_kernel(double *__restrict__ gram, double *__restrict__ diag,
                                                                 double *__restrict__ off, double *__restrict__ tau,
                                                                 const int *__restrict__ list, const int *__restrict__ count) {
     extern __shared__ __align__(16) double td_refl[];   // [D][D]: staging of the matrix, then the reflectors
-    __shared__ __align__(16) double up[2][TD_PLEN];     // u, permuted
-    __shared__ __align__(16) double pp[2][TD_PLEN];     // p, permuted
-    __shared__ __align__(16) double wsum[2][8];
-    __shared__ double sgam[2];
-    __shared__ double s_dg[D], s_of[D], s_ta[D];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    __shared__ __align__(16) TdShared sh;
+    const int tid = threadIdx.x, lane = tid & 31;
     const int tr = tid >> 4, tc = tid & 15;
     int blk = blockIdx.x;
     if (list) {
@@ -50,10 +201,10 @@ __global__ void __launch_bounds__(TD_THREADS, 1) tridiag_kernel(double *__restri
     for (int e = tid; e < D * D / 2; e += TD_THREADS)
         reinterpret_cast<double2 *>(td_refl)[e] = reinterpret_cast<const double2 *>(G)[e];
     if (tid < TD_PLEN) {
-        up[0][tid] = 0.0;
-        up[1][tid] = 0.0;
-        pp[0][tid] = 0.0;
-        pp[1][tid] = 0.0;
+        sh.up[0][tid] = 0.0;
+        sh.up[1][tid] = 0.0;
+        sh.pp[0][tid] = 0.0;
+        sh.pp[1][tid] = 0.0;
     }
     __syncthreads();
     double A[8][8];
@@ -63,165 +214,35 @@ __global__ void __launch_bounds__(TD_THREADS, 1) tridiag_kernel(double *__restri
         for (int b = 0; b < 8; ++b) A[a][b] = td_refl[(tr + 16 * a) * D + tc + 16 * b];
     __syncthreads();
 
-    // The sixteen threads that hold row r publish its tail as the reflector of step r.
-    auto publish = [&](int r, int nxt) {
-        const unsigned mask = 0xFFFFu << (lane & 16);
-        const int ar = r >> 4;
-        double x[8];
-#pragma unroll
-        for (int b = 0; b < 8; ++b) {
-            double v = A[0][b];
-#pragma unroll
-            for (int a = 1; a < 8; ++a) v = (ar == a) ? A[a][b] : v;
-            x[b] = v;
-        }
-        double ss0 = 0.0, ss1 = 0.0, dsel = 0.0;
-#pragma unroll
-        for (int b = 0; b < 8; ++b) {
-            const int j = tc + 16 * b;
-            dsel = (j == r) ? x[b] : dsel;
-            x[b] = (j > r) ? x[b] : 0.0;
-            const double t = (j > r + 1) ? x[b] : 0.0;
-            if (b & 1) ss1 = fma(t, t, ss1);
-            else ss0 = fma(t, t, ss0);
-        }
-        double2 *dst = reinterpret_cast<double2 *>(&up[nxt][tc * TD_PSTRIDE]);
-        dst[0] = make_double2(x[0], x[1]);
-        dst[1] = make_double2(x[2], x[3]);
-        dst[2] = make_double2(x[4], x[5]);
-        dst[3] = make_double2(x[6], x[7]);
-        double ss = ss0 + ss1;
-#pragma unroll
-        for (int o = 8; o > 0; o >>= 1) {
-            ss += __shfl_xor_sync(mask, ss, o);
-            dsel += __shfl_xor_sync(mask, dsel, o);
-        }
-        __syncwarp(mask);
-        const double alpha = up[nxt][td_pos(r + 1)];
-        double beta = alpha, gamma = 0.0;
-        if (ss > 0.0) {
-            const double nrm = sqrt(fma(alpha, alpha, ss));
-            beta = (alpha >= 0.0) ? -nrm : nrm;
-            gamma = 1.0 / (beta * (beta - alpha));
-        }
-        __syncwarp(mask);
-        if (tc == 0) {
-            up[nxt][td_pos(r + 1)] = alpha - beta;
-            sgam[nxt] = gamma;
-            s_dg[r] = dsel;
-            s_of[r] = beta;
-            s_ta[r] = gamma;
-        }
-    };
-
-    if (tr == 0) publish(0, 0);
-
+    if (tr == 0) td_publish<0>(A, 0, 0, tc, lane, sh);
+#pragma unroll 1
     for (int k = 0; k < D - 2; ++k) {
-        __syncthreads();
-        const int cur = k & 1;
-        const double gamma = sgam[cur];
-        if (tid < D) td_refl[k * D + tid] = (tid > k) ? up[cur][td_pos(tid)] : 0.0;
-        if (gamma != 0.0) {   // uniform over the CTA
-            // first live row / column slot of this thread (rows tr + 16 a > k, columns tc + 16 b > k)
-            const int a0 = (k - tr + 16) >> 4, b0 = (k - tc + 16) >> 4;
-            double uj[8], ui[8], acc[8];
-            {
-                const double2 *src = reinterpret_cast<const double2 *>(&up[cur][tc * TD_PSTRIDE]);
-                const double2 v0 = src[0], v1 = src[1], v2 = src[2], v3 = src[3];
-                uj[0] = v0.x; uj[1] = v0.y; uj[2] = v1.x; uj[3] = v1.y;
-                uj[4] = v2.x; uj[5] = v2.y; uj[6] = v3.x; uj[7] = v3.y;
-                const double2 *srow = reinterpret_cast<const double2 *>(&up[cur][tr * TD_PSTRIDE]);
-                const double2 r0 = srow[0], r1 = srow[1], r2 = srow[2], r3 = srow[3];
-                ui[0] = r0.x; ui[1] = r0.y; ui[2] = r1.x; ui[3] = r1.y;
-                ui[4] = r2.x; ui[5] = r2.y; ui[6] = r3.x; ui[7] = r3.y;
-            }
-            double tloc = 0.0;
-#pragma unroll
-            for (int a = 0; a < 8; ++a) {
-                acc[a] = 0.0;
-                if (a >= a0) {
-                    double s0 = 0.0, s1 = 0.0;
-#pragma unroll
-                    for (int b = 0; b < 8; b += 2) {
-                        if (b + 1 >= b0) {
-                            s0 = fma(A[a][b], uj[b], s0);
-                            s1 = fma(A[a][b + 1], uj[b + 1], s1);
-                        }
-                    }
-                    acc[a] = s0 + s1;
-                    tloc = fma(ui[a], acc[a], tloc);
-                }
-            }
-            // sum the partial rows over the sixteen column groups: each stage keeps half of the rows
-            const bool h8 = tc & 8, h4 = tc & 4, h2 = tc & 2;
-            double v4[4], v2[2], v1;
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const double keep = h8 ? acc[q + 4] : acc[q], send = h8 ? acc[q] : acc[q + 4];
-                v4[q] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
-            }
-#pragma unroll
-            for (int q = 0; q < 2; ++q) {
-                const double keep = h4 ? v4[q + 2] : v4[q], send = h4 ? v4[q] : v4[q + 2];
-                v2[q] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
-            }
-            {
-                const double keep = h2 ? v2[1] : v2[0], send = h2 ? v2[0] : v2[1];
-                v1 = keep + __shfl_xor_sync(0xffffffffu, send, 2);
-            }
-            v1 += __shfl_xor_sync(0xffffffffu, v1, 1);
-            const int arow = (h8 ? 4 : 0) + (h4 ? 2 : 0) + (h2 ? 1 : 0);
-            const int irow = tr + 16 * arow;
-            if (!(tc & 1) && irow > k) pp[cur][td_pos(irow)] = gamma * v1;
-            tloc = warp_sum(tloc);
-            if (lane == 0) wsum[cur][warp] = tloc;
-            __syncthreads();
-            const double2 w0 = *reinterpret_cast<const double2 *>(&wsum[cur][0]), w1 = *reinterpret_cast<const double2 *>(&wsum[cur][2]);
-            const double2 w2 = *reinterpret_cast<const double2 *>(&wsum[cur][4]), w3 = *reinterpret_cast<const double2 *>(&wsum[cur][6]);
-            const double uAu = ((w0.x + w0.y) + (w1.x + w1.y)) + ((w2.x + w2.y) + (w3.x + w3.y));
-            const double twoK = gamma * gamma * uAu;
-            double pj[8], si[8];
-            {
-                const double2 *src = reinterpret_cast<const double2 *>(&pp[cur][tc * TD_PSTRIDE]);
-                const double2 v0 = src[0], v1b = src[1], v2b = src[2], v3 = src[3];
-                pj[0] = v0.x; pj[1] = v0.y; pj[2] = v1b.x; pj[3] = v1b.y;
-                pj[4] = v2b.x; pj[5] = v2b.y; pj[6] = v3.x; pj[7] = v3.y;
-                const double2 *srow = reinterpret_cast<const double2 *>(&pp[cur][tr * TD_PSTRIDE]);
-                const double2 r0 = srow[0], r1 = srow[1], r2 = srow[2], r3 = srow[3];
-                si[0] = r0.x; si[1] = r0.y; si[2] = r1.x; si[3] = r1.y;
-                si[4] = r2.x; si[5] = r2.y; si[6] = r3.x; si[7] = r3.y;
-            }
-#pragma unroll
-            for (int a = 0; a < 8; ++a) {
-                if (a >= a0) {
-                    const double s_i = fma(-twoK, ui[a], si[a]), u_i = ui[a];
-#pragma unroll
-                    for (int b = 0; b < 8; b += 2) {
-                        if (b + 1 >= b0) {
-                            A[a][b] = fma(-u_i, pj[b], fma(-s_i, uj[b], A[a][b]));
-                            A[a][b + 1] = fma(-u_i, pj[b + 1], fma(-s_i, uj[b + 1], A[a][b + 1]));
-                        }
-                    }
-                }
-            }
+        switch ((k + 1) >> 4) {
+            case 0: td_step<0>(A, k, tid, sh, td_refl); break;
+            case 1: td_step<1>(A, k, tid, sh, td_refl); break;
+            case 2: td_step<2>(A, k, tid, sh, td_refl); break;
+            case 3: td_step<3>(A, k, tid, sh, td_refl); break;
+            case 4: td_step<4>(A, k, tid, sh, td_refl); break;
+            case 5: td_step<5>(A, k, tid, sh, td_refl); break;
+            case 6: td_step<6>(A, k, tid, sh, td_refl); break;
+            default: td_step<7>(A, k, tid, sh, td_refl); break;
         }
-        if (tr == ((k + 1) & 15) && k + 1 < D - 2) publish(k + 1, cur ^ 1);
     }
-    if (tid == 14 * 16 + 14) s_dg[D - 2] = A[7][7];
-    if (tid == 14 * 16 + 15) s_of[D - 2] = A[7][7];
-    if (tid == 15 * 16 + 15) s_dg[D - 1] = A[7][7];
+    if (tid == 14 * 16 + 14) sh.dg[D - 2] = A[7][7];
+    if (tid == 14 * 16 + 15) sh.of[D - 2] = A[7][7];
+    if (tid == 15 * 16 + 15) sh.dg[D - 1] = A[7][7];
     if (tid == 0) {
-        s_of[D - 1] = 0.0;
-        s_ta[D - 2] = 0.0;
-        s_ta[D - 1] = 0.0;
+        sh.of[D - 1] = 0.0;
+        sh.ta[D - 2] = 0.0;
+        sh.ta[D - 1] = 0.0;
     }
     __syncthreads();
     for (int e = tid; e < (D - 2) * D / 2; e += TD_THREADS)
         reinterpret_cast<double2 *>(G)[e] = reinterpret_cast<const double2 *>(td_refl)[e];
     if (tid < D) {
-        diag[static_cast<size_t>(blk) * D + tid] = s_dg[tid];
-        off[static_cast<size_t>(blk) * D + tid] = s_of[tid];
-        tau[static_cast<size_t>(blk) * D + tid] = s_ta[tid];
+        diag[static_cast<size_t>(blk) * D + tid] = sh.dg[tid];
+        off[static_cast<size_t>(blk) * D + tid] = sh.of[tid];
+        tau[static_cast<size_t>(blk) * D + tid] = sh.ta[tid];
     }
 }
 
