@@ -289,10 +289,22 @@ extern "C" int eosq_scores(eosq_ctx *ctx, const eosq_cache_t *kcache, int64_t nu
     if ((rc = get_rotation(ctx, d, seed, &rot)) != EOSQ_OK) return rc;
     if ((rc = get_codebook(d, bits, &cb)) != EOSQ_OK) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    run_stage(ctx, ST_SCORES, s, [&] {
-        launch_scores_plain(*kcache, num_kv_heads, blocks_per_head, head_stride_blocks, n, rot, cb,
-                            static_cast<const __half *>(q), G, scale, scores, s);
-    });
+    if (scores_tc_supported(bits, n) && (reinterpret_cast<uintptr_t>(kcache->codes) & 15u) == 0) {
+        bool setup_ok = true;
+        run_stage(ctx, ST_SCORES, s, [&] {
+            setup_ok = launch_scores_tc(*kcache, num_kv_heads, blocks_per_head, head_stride_blocks, n, rot, cb,
+                                        static_cast<const __half *>(q), G, scale, scores, ctx->dev_err, ctx->sm_count, s);
+        });
+        if (!setup_ok) {
+            ctx->last_error = "tensor-core score kernel: launch set-up failed";
+            return EOSQ_ERR_CUDA;
+        }
+    } else {
+        run_stage(ctx, ST_SCORES, s, [&] {
+            launch_scores_plain(*kcache, num_kv_heads, blocks_per_head, head_stride_blocks, n, rot, cb,
+                                static_cast<const __half *>(q), G, scale, scores, s);
+        });
+    }
     if (record_cuda(ctx, cudaGetLastError(), "eosq_scores launch")) return EOSQ_ERR_CUDA;
     return EOSQ_OK;
 }
