@@ -21,9 +21,9 @@ using namespace sm100;
 
 constexpr int TC_ERR_SCORES_TIMEOUT = 4;
 
-constexpr int SC_THREADS = 256;           // two groups of four warps, each group works on its own tiles
+constexpr int SC_THREADS = 128;           // one token per thread, one tensor-memory lane per token
 constexpr int SC_NQ = 16;                 // query columns per pass (MMA N)
-constexpr uint32_t SC_TMEM_COLS = 256;    // 128 columns per warp group
+constexpr uint32_t SC_TMEM_COLS = 128;
 constexpr uint32_t SC_COL_A = 0;          // code operand: 64 columns (128 fp16)
 constexpr uint32_t SC_COL_P = 64;         // factor operand: 8 columns (16 fp16)
 constexpr uint32_t SC_COL_D1 = 80;        // 16 columns
@@ -80,9 +80,34 @@ struct ScoresArgs {
     int *err;
 };
 
-__global__ void __launch_bounds__(SC_THREADS, 2) scores_tc_kernel(const ScoresArgs a) {
+// What a thread fetches from global memory for one token of one tile.  The values stay exactly as
+// loaded (nothing here depends on a load's result), so a fetch issued one tile ahead does not
+// stall the thread; they are unpacked when the tile is processed.
+constexpr int SC_PMAX = 12;   // factor rows fetched per token: the rank never exceeds the pilot k = 11
+struct ScTokenData {
+    uint4 c0, c1;               // 128 packed 2-bit codes
+    unsigned short p[SC_PMAX];  // fp16 factor entries, rows below the rank
+    unsigned short rho;         // fp16 row norm
+};
+
+__device__ __forceinline__ void sc_fetch(const ScoresArgs &a, long long gb, int rank, int tok, ScTokenData &t) {
+    const bool valid = tok < a.n;
+    const int tk = valid ? tok : 0;
+    const uint4 *src = reinterpret_cast<const uint4 *>(a.cache.codes + (static_cast<size_t>(gb) * a.n + tk) * 32);
+    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+    t.c0 = valid ? __ldg(src) : zero;
+    t.c1 = valid ? __ldg(src + 1) : zero;
+    t.rho = valid ? __ldg(a.cache.norms + static_cast<size_t>(gb) * a.n + tk) : static_cast<unsigned short>(0);
+    const unsigned short *prow = a.cache.P + static_cast<size_t>(gb) * RMAX * a.n + tk;
+#pragma unroll
+    for (int i = 0; i < SC_PMAX; ++i) t.p[i] = (valid && i < rank) ? __ldg(prow + static_cast<size_t>(i) * a.n) : static_cast<unsigned short>(0);
+}
+
+// One CTA of four warps works through a contiguous range of (head, block) items; four CTAs share
+// an SM.  Everything a tile needs from global memory is fetched one tile ahead into registers.
+__global__ void __launch_bounds__(SC_THREADS, 4) scores_tc_kernel(const ScoresArgs a) {
     extern __shared__ uint8_t sc_smem_raw[];
-    __shared__ __align__(8) uint64_t done_bar[2];
+    __shared__ __align__(8) uint64_t done_bar;
     __shared__ uint32_t tmem_base_s;
     __shared__ volatile int abort_flag;
 
@@ -92,13 +117,11 @@ __global__ void __launch_bounds__(SC_THREADS, 2) scores_tc_kernel(const ScoresAr
     float *qs = reinterpret_cast<float *>(base + 12288);    // [16][128] queries of the current head
     __half *vs = reinterpret_cast<__half *>(base + 20480);  // [16][128] right vectors of the current block
     const int tid = threadIdx.x, warp = tid >> 5;
-    const int wg = tid >> 7, wt = tid & 127, lw = warp & 3;
     const int n = a.n, tiles = (n + 127) / 128;
     const int gcount = min(SC_NQ, a.G - a.g0);
 
     if (tid == 0) {
-        mbar_init(&done_bar[0], 1);
-        mbar_init(&done_bar[1], 1);
+        mbar_init(&done_bar, 1);
         abort_flag = 0;
         fence_mbar_init();
     }
@@ -109,8 +132,8 @@ __global__ void __launch_bounds__(SC_THREADS, 2) scores_tc_kernel(const ScoresAr
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    const uint32_t tmem_wg = tmem_base_s + 128u * wg;                                  // lane 0 view (MMA operands)
-    const uint32_t tmem_me = tmem_wg + (static_cast<uint32_t>(32 * lw) << 16);           // this warp's lanes
+    const uint32_t tmem0 = tmem_base_s;                                           // lane 0 view (MMA operands)
+    const uint32_t tmem_me = tmem0 + (static_cast<uint32_t>(32 * warp) << 16);    // this warp's lanes
 
     const long long ipc = (a.items + gridDim.x - 1) / gridDim.x;
     const long long it0 = ipc * blockIdx.x, it1 = min(a.items, it0 + ipc);
@@ -118,45 +141,86 @@ __global__ void __launch_bounds__(SC_THREADS, 2) scores_tc_kernel(const ScoresAr
     uint32_t done_cnt = 0;
     constexpr uint32_t idesc = umma_idesc_f16(128, SC_NQ, false, false);
 
+    auto block_of = [&](long long item) { return (item / a.bph) * a.head_stride + (item % a.bph); };
+    // prefetch state: the next tile's token data, the next block's rank and right vectors
+    ScTokenData nxt;
+    int rank = 0, rank_next = 0;
+    uint4 v_next[2];
+    if (it0 < it1) {
+        const long long gb0 = block_of(it0);
+        rank = __ldg(a.cache.rank + gb0);
+        const uint4 *vsrc = reinterpret_cast<const uint4 *>(a.cache.V + gb0 * RMAX * D);
+        v_next[0] = __ldg(vsrc + tid);
+        v_next[1] = __ldg(vsrc + SC_THREADS + tid);
+        sc_fetch(a, gb0, rank, tid, nxt);
+    }
+
     for (long long item = it0; item < it1; ++item) {
         const long long head = item / a.bph, jb = item % a.bph;
-        const long long gb = head * a.head_stride + jb;
+        const long long gb = block_of(item);
+        __syncthreads();   // the previous block's MMAs have been waited for: the shared operands are free
+        if (abort_flag) break;
         if (head != cur_head) {
-            __syncthreads();
             for (int e = tid; e < SC_NQ * D; e += SC_THREADS) {
                 const int g = e / D;
                 qs[e] = (g < gcount) ? __half2float(a.q[(head * a.G + a.g0 + g) * D + (e % D)]) : 0.0f;
             }
             __syncthreads();
-            const int c = tid & (D - 1), half = tid >> 7;
-            float w[8];
+            const int c = tid;   // SC_THREADS == D
+            float w[SC_NQ];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) w[i] = 0.0f;
+            for (int i = 0; i < SC_NQ; ++i) w[i] = 0.0f;
             for (int j = 0; j < D; ++j) {
                 const float pv = a.pi_t[j * D + c];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) w[i] = fmaf(pv, qs[(8 * half + i) * D + j], w[i]);
+                for (int i = 0; i < SC_NQ; ++i) w[i] = fmaf(pv, qs[i * D + j], w[i]);
             }
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
+            for (int i = 0; i < SC_NQ; ++i) {
                 __half hi, lo;
                 sc_split(w[i] * SC_QSCALE, hi, lo);
-                const uint32_t off = sc_b_offset(8 * half + i, c, SC_NQ);
+                const uint32_t off = sc_b_offset(i, c, SC_NQ);
                 *reinterpret_cast<__half *>(b1_hi + off) = hi;
                 *reinterpret_cast<__half *>(b1_lo + off) = lo;
             }
             cur_head = head;
         }
-        const int rank = a.cache.rank[gb];
-        reinterpret_cast<uint4 *>(vs)[tid] = reinterpret_cast<const uint4 *>(a.cache.V + gb * RMAX * D)[tid];
-        __syncthreads();   // every group is past the previous block; vs and qs are in place
-        if (abort_flag) break;
-        {
-            const int g = tid >> 4, i = tid & 15;
+        reinterpret_cast<uint4 *>(vs)[tid] = v_next[0];
+        reinterpret_cast<uint4 *>(vs)[SC_THREADS + tid] = v_next[1];
+        const bool more = item + 1 < it1;
+        const long long gb_next = more ? block_of(item + 1) : gb;
+        if (more) {
+            rank_next = __ldg(a.cache.rank + gb_next);
+            const uint4 *vsrc = reinterpret_cast<const uint4 *>(a.cache.V + gb_next * RMAX * D);
+            v_next[0] = __ldg(vsrc + tid);
+            v_next[1] = __ldg(vsrc + SC_THREADS + tid);
+        }
+        __syncthreads();
+        for (int e = tid; e < SC_NQ * RMAX; e += SC_THREADS) {   // Aq[g][i] = q_g . zeta_i
+            const int g = e >> 4, i = e & 15;
             float dot = 0.0f;
-            if (i < rank) {
-#pragma unroll 8
-                for (int j = 0; j < D; ++j) dot = fmaf(qs[g * D + j], __half2float(vs[i * D + j]), dot);
+            if (i < rank && g < gcount) {
+                const uint4 *vrow = reinterpret_cast<const uint4 *>(vs + i * D);
+                const float4 *qrow = reinterpret_cast<const float4 *>(qs + g * D);
+                float d0 = 0.0f, d1 = 0.0f;
+#pragma unroll 4
+                for (int j = 0; j < D / 8; ++j) {
+                    const uint4 v = vrow[j];
+                    const float4 qa = qrow[2 * j], qb = qrow[2 * j + 1];
+                    const float2 v0 = __half22float2(*reinterpret_cast<const __half2 *>(&v.x));
+                    const float2 v1 = __half22float2(*reinterpret_cast<const __half2 *>(&v.y));
+                    const float2 v2 = __half22float2(*reinterpret_cast<const __half2 *>(&v.z));
+                    const float2 v3 = __half22float2(*reinterpret_cast<const __half2 *>(&v.w));
+                    d0 = fmaf(qa.x, v0.x, d0);
+                    d1 = fmaf(qa.y, v0.y, d1);
+                    d0 = fmaf(qa.z, v1.x, d0);
+                    d1 = fmaf(qa.w, v1.y, d1);
+                    d0 = fmaf(qb.x, v2.x, d0);
+                    d1 = fmaf(qb.y, v2.y, d1);
+                    d0 = fmaf(qb.z, v3.x, d0);
+                    d1 = fmaf(qb.w, v3.y, d1);
+                }
+                dot = d0 + d1;
             }
             __half hi, lo;
             sc_split(dot * SC_QSCALE, hi, lo);
@@ -167,58 +231,49 @@ __global__ void __launch_bounds__(SC_THREADS, 2) scores_tc_kernel(const ScoresAr
         fence_proxy_async_smem();
         __syncthreads();
 
-        for (int tile = wg; tile < tiles; tile += 2) {
-            const int tok = tile * 128 + wt;
-            const bool valid = tok < n;
-            uint32_t cw[8];
-            float rho = 0.0f;
-            uint32_t pw[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                cw[i] = 0u;
-                pw[i] = 0u;
-            }
-            if (valid) {
-                const uint4 *src = reinterpret_cast<const uint4 *>(a.cache.codes + (static_cast<size_t>(gb) * n + tok) * 32);
-                const uint4 c0 = src[0], c1 = src[1];
-                cw[0] = c0.x; cw[1] = c0.y; cw[2] = c0.z; cw[3] = c0.w;
-                cw[4] = c1.x; cw[5] = c1.y; cw[6] = c1.z; cw[7] = c1.w;
-                rho = __half2float(__ushort_as_half(a.cache.norms[static_cast<size_t>(gb) * n + tok]));
-#pragma unroll
-                for (int i = 0; i < RMAX; ++i) {
-                    if (i < rank) {
-                        const uint32_t v = a.cache.P[(static_cast<size_t>(gb) * RMAX + i) * n + tok];
-                        pw[i >> 1] |= v << (16 * (i & 1));
-                    }
-                }
-            }
+        bool ok = true;
+        for (int tile = 0; tile < tiles; ++tile) {
+            const ScTokenData cur = nxt;
+            const int tok = tile * 128 + tid;
+            if (tile + 1 < tiles) sc_fetch(a, gb, rank, tok + 128, nxt);
+            else if (more) sc_fetch(a, gb_next, rank_next, tid, nxt);
             {
                 uint32_t av[32];
 #pragma unroll
-                for (int q = 0; q < 4; ++q) sc_expand16(cw[q], a.lo_tab, a.hi_tab, &av[8 * q]);
+                const uint32_t w0[4] = {cur.c0.x, cur.c0.y, cur.c0.z, cur.c0.w}, w1[4] = {cur.c1.x, cur.c1.y, cur.c1.z, cur.c1.w};
+#pragma unroll
+                for (int q = 0; q < 4; ++q) sc_expand16(w0[q], a.lo_tab, a.hi_tab, &av[8 * q]);
                 tmem_st32(tmem_me + SC_COL_A, av);
 #pragma unroll
-                for (int q = 0; q < 4; ++q) sc_expand16(cw[4 + q], a.lo_tab, a.hi_tab, &av[8 * q]);
+                for (int q = 0; q < 4; ++q) sc_expand16(w1[q], a.lo_tab, a.hi_tab, &av[8 * q]);
                 tmem_st32(tmem_me + SC_COL_A + 32, av);
             }
-            tmem_st8(tmem_me + SC_COL_P, pw);
+            {
+                uint32_t pw[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const uint32_t lo = (2 * i < SC_PMAX) ? cur.p[2 * i] : 0u, hi = (2 * i + 1 < SC_PMAX) ? cur.p[2 * i + 1] : 0u;
+                    pw[i] = lo | (hi << 16);
+                }
+                tmem_st8(tmem_me + SC_COL_P, pw);
+            }
             tmem_st_wait();
             tc_fence_before_sync();
-            asm volatile("bar.sync %0, %1;" ::"r"(1 + wg), "r"(128) : "memory");
-            if (wt == 0) {
+            __syncthreads();
+            if (tid == 0) {
                 tc_fence_after_sync();
                 const uint32_t h1 = smem_u32(b1_hi), l1 = smem_u32(b1_lo);
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
                     const uint32_t kb = (ks >> 2) * (SC_NQ * 128) + (ks & 3) * 32;
-                    umma_f16_ts(tmem_wg + SC_COL_D1, tmem_wg + SC_COL_A + 8 * ks, umma_desc_sw128(h1 + kb, 16, 1024), idesc, ks ? 1u : 0u);
-                    umma_f16_ts(tmem_wg + SC_COL_D1, tmem_wg + SC_COL_A + 8 * ks, umma_desc_sw128(l1 + kb, 16, 1024), idesc, 1u);
+                    umma_f16_ts(tmem0 + SC_COL_D1, tmem0 + SC_COL_A + 8 * ks, umma_desc_sw128(h1 + kb, 16, 1024), idesc, ks ? 1u : 0u);
+                    umma_f16_ts(tmem0 + SC_COL_D1, tmem0 + SC_COL_A + 8 * ks, umma_desc_sw128(l1 + kb, 16, 1024), idesc, 1u);
                 }
-                umma_f16_ts(tmem_wg + SC_COL_D2, tmem_wg + SC_COL_P, umma_desc_sw128(smem_u32(b2_hi), 16, 1024), idesc, 0u);
-                umma_f16_ts(tmem_wg + SC_COL_D2, tmem_wg + SC_COL_P, umma_desc_sw128(smem_u32(b2_lo), 16, 1024), idesc, 1u);
-                umma_commit(&done_bar[wg]);
+                umma_f16_ts(tmem0 + SC_COL_D2, tmem0 + SC_COL_P, umma_desc_sw128(smem_u32(b2_hi), 16, 1024), idesc, 0u);
+                umma_f16_ts(tmem0 + SC_COL_D2, tmem0 + SC_COL_P, umma_desc_sw128(smem_u32(b2_lo), 16, 1024), idesc, 1u);
+                umma_commit(&done_bar);
             }
-            const bool ok = mbar_wait(&done_bar[wg], done_cnt & 1u, &abort_flag);
+            ok = mbar_wait(&done_bar, done_cnt & 1u, &abort_flag);
             done_cnt += 1;
             if (!ok) break;
             tc_fence_after_sync();
@@ -226,16 +281,17 @@ __global__ void __launch_bounds__(SC_THREADS, 2) scores_tc_kernel(const ScoresAr
             tmem_ld16(tmem_me + SC_COL_D1, d1);
             tmem_ld16(tmem_me + SC_COL_D2, d2);
             tmem_ld_wait();
-            if (valid) {
-                const float f1 = a.scale * rho * a.inv_code, f2 = a.scale * (1.0f / SC_QSCALE);
+            if (tok < n) {
+                const float f1 = a.scale * __half2float(__ushort_as_half(cur.rho)) * a.inv_code, f2 = a.scale * (1.0f / SC_QSCALE);
                 float *dst = a.scores + (head * a.G + a.g0) * (a.bph * n) + jb * n + tok;
 #pragma unroll
                 for (int g = 0; g < SC_NQ; ++g)
                     if (g < gcount) dst[static_cast<size_t>(g) * (a.bph * n)] = fmaf(f1, __uint_as_float(d1[g]), f2 * __uint_as_float(d2[g]));
             }
             tc_fence_before_sync();
-            asm volatile("bar.sync %0, %1;" ::"r"(1 + wg), "r"(128) : "memory");
+            __syncthreads();
         }
+        rank = rank_next;
     }
 
     __syncthreads();
@@ -303,7 +359,7 @@ bool launch_scores_tc(const eosq_cache_t &cache, int64_t heads, int64_t bph, int
     a.q = q;
     a.scores = scores;
     a.err = err;
-    const int grid = static_cast<int>(std::min<int64_t>(a.items, 2 * static_cast<int64_t>(sm_count)));
+    const int grid = static_cast<int>(std::min<int64_t>(a.items, 4 * static_cast<int64_t>(sm_count)));
     for (int g0 = 0; g0 < G; g0 += SC_NQ) {
         a.g0 = g0;
         scores_tc_kernel<<<grid, SC_THREADS, smem, s>>>(a);

@@ -46,6 +46,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
     for (uint32_t it = 0; it < WAIT_POLLS; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 63u) == 63u && *abort_flag) return false;
+        if (it >= 2) __nanosleep(it < 16 ? 64 : 256);   // back off: a spinning warp steals issue slots from working ones
     }
     *abort_flag = 1;
     return false;
