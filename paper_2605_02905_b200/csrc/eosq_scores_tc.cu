@@ -305,7 +305,7 @@ __global__ void __launch_bounds__(SC_THREADS, 4) scores_tc_kernel(const ScoresAr
 // Scale factor kappa in [8, 16) for which the fp16 roundings of kappa * centroid are, jointly, as
 // close to exact as possible (searched over 4096 mantissas); with four levels the worst relative
 // rounding error drops from 2.4e-4 to the 1e-6 range.
-static float best_table_scale(const Codebook &cb, uint16_t (&table)[16]) {
+float best_table_scale(const Codebook &cb, uint16_t (&table)[16]) {
     const int levels = 1 << cb.bits;
     double best_err = 1e30;
     float best = 8.0f;
@@ -326,6 +326,11 @@ static float best_table_scale(const Codebook &cb, uint16_t (&table)[16]) {
     return best;
 }
 
+bool scores_ws_supported(const eosq_cache_t &cache, int bits, int n);
+bool launch_scores_ws(const eosq_cache_t &cache, int64_t heads, int64_t bph, int64_t head_stride, int n, const Rotation &rot,
+                      const uint16_t (&table)[16], float kappa, const __half *q, int G, float scale, float *scores, int *err,
+                      int sm_count, cudaStream_t s);
+
 bool scores_tc_supported(int bits, int n) { return bits == 2 && n >= 128; }
 
 bool launch_scores_tc(const eosq_cache_t &cache, int64_t heads, int64_t bph, int64_t head_stride, int n, const Rotation &rot,
@@ -338,8 +343,16 @@ bool launch_scores_tc(const eosq_cache_t &cache, int64_t heads, int64_t bph, int
             return false;
         configured = true;
     }
-    uint16_t table[16];
-    const float kappa = best_table_scale(cb, table);
+    // the table depends only on the codebook: search once per bit width
+    static uint16_t table[16];
+    static float kappa = 0.0f;
+    static int table_bits = 0;
+    if (table_bits != cb.bits) {
+        kappa = best_table_scale(cb, table);
+        table_bits = cb.bits;
+    }
+    if (scores_ws_supported(cache, cb.bits, n))
+        return launch_scores_ws(cache, heads, bph, head_stride, n, rot, table, kappa, q, G, scale, scores, err, sm_count, s);
     ScoresArgs a;
     a.cache = cache;
     a.bph = bph;

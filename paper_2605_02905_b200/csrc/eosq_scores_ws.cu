@@ -1,0 +1,548 @@
+// Warp-specialised attention-logit kernel for 2-bit codes (Remark 6.4): one persistent CTA of 16
+// warps per SM in which loading, code expansion, the MMAs and the output run concurrently on
+// different tiles.
+//
+//   warp 0        bulk-copies each 128-token tile (codes, norms, factor rows) and each block's right
+//                 vectors from global memory into a ring of shared-memory stages
+//   warps 2-3     build the query-side operands: W = Pi q once per head, Aq = q V^T once per block
+//   warps 4-11    two groups of four: expand a tile's codes to fp16 centroids (byte permutes) and
+//                 store them, the factor entries and the row norm into one of four tensor-memory
+//                 buffers, one token per thread
+//   warp 1        issues the nine MMAs of a tile (A from tensor memory, B from shared memory)
+//   warps 12-15   read the accumulators back, apply norm and scale, write the logits
+//
+// The high and the low fp16 plane of a query-side operand are stacked along N (columns g and
+// 8 + g of one 16-column accumulator), so a pass serves eight query vectors.
+#include <algorithm>
+
+#include "eosq_common.cuh"
+#include "eosq_sm100.cuh"
+
+namespace eosq {
+
+using namespace sm100;
+
+constexpr int TC_ERR_SCORES_WS_TIMEOUT = 8;
+
+constexpr int WS_THREADS = 512;
+constexpr int WS_NQ = 8;                   // query vectors per pass
+constexpr int WS_STAGES = 5;               // shared-memory stages of WS_TPS tiles each
+constexpr int WS_TPS = 4;                  // tiles per stage: few large copies keep the copy engine's queue short
+constexpr int WS_BUFS = 4;
+constexpr int WS_PMAX = 12;                // factor rows staged per tile (rank <= pilot k = 11)
+constexpr uint32_t WS_ST_CODES = 0, WS_ST_NORMS = 16384, WS_ST_P = 17408;   // 512 tokens: codes, norms, 2 boxes of 12 x 256 factors
+constexpr uint32_t WS_ST_PBOX = WS_PMAX * 512;
+constexpr uint32_t WS_STAGE_BYTES = WS_ST_P + 2 * WS_ST_PBOX;              // 29696
+constexpr uint32_t WS_TMEM_COLS = 512;
+constexpr uint32_t WS_BUF_COLS = 112;      // per buffer: A 0-63, P 64-71, rho 72, D1 80-95, D2 96-111
+constexpr uint32_t WS_COL_P = 64, WS_COL_RHO = 72, WS_COL_D1 = 80, WS_COL_D2 = 96;
+constexpr float WS_QSCALE = 256.0f;
+
+// shared-memory map (offsets from a 1024-byte aligned base)
+constexpr uint32_t WS_OFF_STAGES = 0;
+constexpr uint32_t WS_OFF_B1 = WS_STAGES * WS_STAGE_BYTES;          // 2 x 4096: W, hi rows 0-7, lo rows 8-15
+constexpr uint32_t WS_OFF_B2 = WS_OFF_B1 + 2 * 4096;                // 2 x 2048: Aq
+constexpr uint32_t WS_OFF_V = WS_OFF_B2 + 2 * 2048;                 // 2 x 4096: right vectors (fp16)
+constexpr uint32_t WS_OFF_Q = WS_OFF_V + 2 * 4096;                  // 2 x (8 x 128) fp32 queries, by head parity
+constexpr uint32_t WS_SMEM_BYTES = WS_OFF_Q + 2 * WS_NQ * D * 4 + 1024;
+
+struct WsArgs {
+    eosq_cache_t cache;
+    int bph, head_stride, heads;   // blocks per head, block stride between heads, heads
+    int n, G, g0;
+    float scale, inv_code;
+    uint32_t lo_tab, hi_tab;
+    const float *pi_t;
+    const __half *q;
+    float *scores;
+    int *err;
+};
+
+__device__ __forceinline__ void ws_bulk_load(void *smem_dst, const void *gsrc, uint32_t bytes, uint64_t *bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :
+                 : "r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(gsrc)), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
+
+__device__ __forceinline__ uint32_t ws_prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+
+// Sixteen 2-bit codes (one word) -> eight words of fp16 pairs through the four-entry byte tables.
+__device__ __forceinline__ void ws_expand16(uint32_t w, uint32_t lo_tab, uint32_t hi_tab, uint32_t *out) {
+#pragma unroll
+    for (int part = 0; part < 2; ++part) {
+        uint32_t t = (w >> (16 * part)) & 0xFFFFu;
+        t = (t | (t << 8)) & 0x00FF00FFu;
+        t = (t | (t << 4)) & 0x0F0F0F0Fu;
+        t = (t | (t << 2)) & 0x33333333u;   // one nibble per code
+#pragma unroll
+        for (int quad = 0; quad < 2; ++quad) {
+            const uint32_t sel = t >> (16 * quad);
+            const uint32_t lows = ws_prmt(lo_tab, 0u, sel), highs = ws_prmt(hi_tab, 0u, sel);
+            out[4 * part + 2 * quad] = ws_prmt(lows, highs, 0x5140u);
+            out[4 * part + 2 * quad + 1] = ws_prmt(lows, highs, 0x7362u);
+        }
+    }
+}
+
+// Byte offset of element (row, k) of a K-major, 128-byte-swizzled operand with 16 rows per 64-wide K box.
+__device__ __forceinline__ uint32_t ws_b_offset(int row, int k) {
+    const int box = k >> 6, kk = k & 63;
+    return box * 2048 + row * 128 + ((((kk >> 3) ^ (row & 7)) << 4) | ((kk & 7) << 1));
+}
+
+__device__ __forceinline__ void ws_split_store(uint8_t *plane, int g, int k, float v) {
+    const __half hi = __float2half_rn(v), lo = __float2half_rn(v - __half2float(hi));
+    *reinterpret_cast<__half *>(plane + ws_b_offset(g, k)) = hi;
+    *reinterpret_cast<__half *>(plane + ws_b_offset(WS_NQ + g, k)) = lo;
+}
+
+struct WsBarriers {
+    uint64_t st_full[WS_STAGES], st_empty[WS_STAGES];
+    uint64_t a_full[WS_BUFS], a_empty[WS_BUFS], d_full[WS_BUFS], d_empty[WS_BUFS];
+    uint64_t blk_full[2], blk_empty[2], b2_full[2], b2_empty[2], b1_full[2], b1_empty[2];
+};
+
+bool make_factor_tensor_map(const void *P, int64_t nb, int n, int rows, CUtensorMap *out);
+
+__global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a, const __grid_constant__ CUtensorMap pmap4,
+                                                                  const __grid_constant__ CUtensorMap pmap8,
+                                                                  const __grid_constant__ CUtensorMap pmap12) {
+    extern __shared__ uint8_t ws_smem_raw[];
+    __shared__ __align__(8) WsBarriers bars;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int st_rank[WS_STAGES];
+    __shared__ volatile int abort_flag;
+
+    uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(ws_smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n = a.n, tiles = (n + 127) / 128;
+    const int gcount = min(WS_NQ, a.G - a.g0);
+
+    if (tid == 0) {
+        for (int s = 0; s < WS_STAGES; ++s) {
+            mbar_init(&bars.st_full[s], 1);
+            mbar_init(&bars.st_empty[s], 128 * WS_TPS);
+        }
+        for (int b = 0; b < WS_BUFS; ++b) {
+            mbar_init(&bars.a_full[b], 128);
+            mbar_init(&bars.a_empty[b], 1);
+            mbar_init(&bars.d_full[b], 1);
+            mbar_init(&bars.d_empty[b], 128);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&bars.blk_full[b], 1);
+            mbar_init(&bars.blk_empty[b], 1);
+            mbar_init(&bars.b2_full[b], 1);
+            mbar_init(&bars.b2_empty[b], 1);
+            mbar_init(&bars.b1_full[b], 1);
+            mbar_init(&bars.b1_empty[b], 1);
+        }
+        abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(&tmem_base_s, WS_TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem0 = tmem_base_s;
+
+    // contiguous range of (head, block) items of this CTA; every role walks it in the same order
+    const int items = a.heads * a.bph;
+    const int ipc = (items + gridDim.x - 1) / gridDim.x;
+    const int it0 = min(items, ipc * static_cast<int>(blockIdx.x)), it1 = min(items, it0 + ipc);
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- loader
+        // Lane 0 keeps the protocol (waits, expected byte counts) and fetches the factor rows of a tile with
+        // one tensor copy (4, 8 or 12 rows, whichever covers the rank); lane 30 copies the codes, lane 31
+        // the norms.
+        if (it0 < it1) {
+            uint32_t sseq = 0;
+            int head = it0 / a.bph, jb = it0 - head * a.bph;
+            int rank_next = min(__ldg(a.cache.rank + static_cast<long long>(head) * a.head_stride + jb), WS_PMAX);
+            bool alive = true;
+            for (int item = it0, bi = 0; item < it1 && alive; ++item, ++bi) {
+                const long long gb = static_cast<long long>(head) * a.head_stride + jb;
+                const int rank = rank_next;
+                int nhead = head, njb = jb + 1;
+                if (njb == a.bph) {
+                    njb = 0;
+                    nhead += 1;
+                }
+                if (item + 1 < it1) rank_next = min(__ldg(a.cache.rank + static_cast<long long>(nhead) * a.head_stride + njb), WS_PMAX);
+                const int vb = bi & 1;
+                if (lane == 0) {
+                    alive = mbar_wait(&bars.blk_empty[vb], ((bi >> 1) & 1u) ^ 1u, &abort_flag);
+                    if (alive) {
+                        mbar_arrive_expect_tx(&bars.blk_full[vb], 4096);
+                        ws_bulk_load(base + WS_OFF_V + vb * 4096, a.cache.V + gb * RMAX * D, 4096, &bars.blk_full[vb]);
+                    }
+                }
+                alive = __shfl_sync(0xffffffffu, alive, 0);
+                for (int tile = 0; tile < tiles && alive; tile += WS_TPS, ++sseq) {
+                    const int stage = sseq % WS_STAGES;
+                    const int tok0 = tile * 128;
+                    const uint32_t rows = static_cast<uint32_t>(min(128 * WS_TPS, n - tok0));
+                    const uint32_t boxes = (rows + 255u) >> 8;
+                    const int r4 = (rank + 3) >> 2;
+                    if (lane == 0) {
+                        alive = mbar_wait(&bars.st_empty[stage], ((sseq / WS_STAGES) & 1u) ^ 1u, &abort_flag);
+                        if (alive) {
+                            st_rank[stage] = rank;
+                            mbar_arrive_expect_tx(&bars.st_full[stage], rows * 34u + boxes * static_cast<uint32_t>(r4) * 2048u);
+                        }
+                    }
+                    alive = __shfl_sync(0xffffffffu, alive, 0);
+                    if (!alive) break;
+                    uint8_t *st = base + WS_OFF_STAGES + stage * WS_STAGE_BYTES;
+                    const size_t t0 = static_cast<size_t>(gb) * n + tok0;
+                    if (lane < 2) {
+                        if (r4 > 0 && static_cast<uint32_t>(lane) < boxes)
+                            tma_load_3d(st + WS_ST_P + lane * WS_ST_PBOX, r4 == 1 ? &pmap4 : (r4 == 2 ? &pmap8 : &pmap12), &bars.st_full[stage],
+                                        tok0 + 256 * lane, 0, static_cast<int>(gb));
+                    } else if (lane == 30)
+                        ws_bulk_load(st + WS_ST_CODES, a.cache.codes + t0 * 32, rows * 32, &bars.st_full[stage]);
+                    else if (lane == 31)
+                        ws_bulk_load(st + WS_ST_NORMS, a.cache.norms + t0, rows * 2, &bars.st_full[stage]);
+                }
+                head = nhead;
+                jb = njb;
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issue
+        if (lane == 0 && it0 < it1) {
+            constexpr uint32_t idesc = umma_idesc_f16(128, 16, false, false);
+            uint32_t seq = 0;
+            int head = it0 / a.bph, jb = it0 - head * a.bph, hidx = -1, prev_head = -1;
+            bool alive = true;
+            for (int item = it0, bi = 0; item < it1 && alive; ++item, ++bi) {
+                if (head != prev_head) {
+                    hidx += 1;
+                    prev_head = head;
+                    if (!mbar_wait(&bars.b1_full[hidx & 1], (hidx >> 1) & 1u, &abort_flag)) break;
+                }
+                const int vb = bi & 1, hb = hidx & 1;
+                if (!mbar_wait(&bars.b2_full[vb], (bi >> 1) & 1u, &abort_flag)) break;
+                const uint32_t b1 = smem_u32(base + WS_OFF_B1 + hb * 4096), b2 = smem_u32(base + WS_OFF_B2 + vb * 2048);
+                uint64_t bdesc[D / 16 + 1];
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) bdesc[ks] = umma_desc_sw128(b1 + (ks >> 2) * 2048 + (ks & 3) * 32, 16, 1024);
+                bdesc[D / 16] = umma_desc_sw128(b2, 16, 1024);
+                for (int tile = 0; tile < tiles; ++tile, ++seq) {
+                    const int buf = seq & (WS_BUFS - 1);
+                    const uint32_t u = (seq >> 2) & 1u;
+                    if (!mbar_wait(&bars.a_full[buf], u, &abort_flag) || !mbar_wait(&bars.d_empty[buf], u ^ 1u, &abort_flag)) {
+                        alive = false;
+                        break;
+                    }
+                    tc_fence_after_sync();
+                    const uint32_t tb = tmem0 + buf * WS_BUF_COLS;
+#pragma unroll
+                    for (int ks = 0; ks < D / 16; ++ks) umma_f16_ts(tb + WS_COL_D1, tb + 8 * ks, bdesc[ks], idesc, ks ? 1u : 0u);
+                    umma_f16_ts(tb + WS_COL_D2, tb + WS_COL_P, bdesc[D / 16], idesc, 0u);
+                    umma_commit(&bars.d_full[buf]);
+                    umma_commit(&bars.a_empty[buf]);
+                }
+                if (!alive) break;
+                umma_commit(&bars.b2_empty[vb]);
+                int nhead = head, njb = jb + 1;
+                if (njb == a.bph) {
+                    njb = 0;
+                    nhead += 1;
+                }
+                if (nhead != head || item + 1 == it1) umma_commit(&bars.b1_empty[hb]);
+                head = nhead;
+                jb = njb;
+            }
+        }
+    } else if (warp < 4) {
+        // ---------------------------------------------------------------- operand builder (64 threads)
+        const int bt = tid - 64;
+        float *qs_all = reinterpret_cast<float *>(base + WS_OFF_Q);
+        // W = Pi q of head `hd`, the `hx`-th head of this CTA, into the operand buffer of its parity
+        auto build_w = [&](int hd, int hx) -> bool {
+            const int hb = hx & 1;
+            float *qs = qs_all + hb * WS_NQ * D;
+            if (!mbar_wait(&bars.b1_empty[hb], ((hx >> 1) & 1u) ^ 1u, &abort_flag)) return false;
+            for (int e = bt; e < WS_NQ * D; e += 64) {
+                const int g = e / D;
+                qs[e] = (g < gcount) ? __half2float(a.q[(static_cast<long long>(hd) * a.G + a.g0 + g) * D + (e % D)]) : 0.0f;
+            }
+            asm volatile("bar.sync 2, 64;" ::: "memory");
+            uint8_t *b1 = base + WS_OFF_B1 + hb * 4096;
+            for (int rep = 0; rep < 2; ++rep) {
+                const int c = bt + 64 * rep;
+                float w[WS_NQ];
+#pragma unroll
+                for (int g = 0; g < WS_NQ; ++g) w[g] = 0.0f;
+#pragma unroll 1
+                for (int j0 = 0; j0 < D; j0 += 32) {
+                    float pv[32];
+#pragma unroll
+                    for (int jj = 0; jj < 32; ++jj) pv[jj] = __ldg(a.pi_t + (j0 + jj) * D + c);   // 32 loads in flight
+#pragma unroll
+                    for (int jj = 0; jj < 32; ++jj) {
+#pragma unroll
+                        for (int g = 0; g < WS_NQ; ++g) w[g] = fmaf(pv[jj], qs[g * D + j0 + jj], w[g]);
+                    }
+                }
+#pragma unroll
+                for (int g = 0; g < WS_NQ; ++g) ws_split_store(b1, g, c, w[g] * WS_QSCALE);
+            }
+            fence_proxy_async_smem();
+            asm volatile("bar.sync 2, 64;" ::: "memory");
+            if (bt == 0) mbar_arrive(&bars.b1_full[hb]);
+            return true;
+        };
+        int head = (it0 < it1) ? it0 / a.bph : 0, jb = it0 - head * a.bph, hidx = -1, prev_head = -1;
+        bool first_of_head = false;
+        for (int item = it0, bi = 0; item < it1; ++item, ++bi) {
+            if (head != prev_head) {
+                hidx += 1;
+                prev_head = head;
+                first_of_head = true;
+                if (hidx == 0 && !build_w(head, 0)) break;   // later heads were built one head ahead (below)
+            }
+            const float *qs = qs_all + (hidx & 1) * WS_NQ * D;
+            const long long gb = static_cast<long long>(head) * a.head_stride + jb;
+            const int vb = bi & 1;
+            const int rank = min(__ldg(a.cache.rank + gb), WS_PMAX);
+            if (!mbar_wait(&bars.blk_full[vb], (bi >> 1) & 1u, &abort_flag) ||
+                !mbar_wait(&bars.b2_empty[vb], ((bi >> 1) & 1u) ^ 1u, &abort_flag))
+                break;
+            const __half *vs = reinterpret_cast<const __half *>(base + WS_OFF_V + vb * 4096);
+            uint8_t *b2 = base + WS_OFF_B2 + vb * 2048;
+            for (int e = bt; e < WS_NQ * RMAX; e += 64) {   // Aq[g][i] = q_g . zeta_i
+                const int g = e >> 4, i = e & 15;
+                float dot = 0.0f;
+                if (i < rank && g < gcount) {
+                    const uint4 *vrow = reinterpret_cast<const uint4 *>(vs + i * D);
+                    const float4 *qrow = reinterpret_cast<const float4 *>(qs + g * D);
+                    float d0 = 0.0f, d1 = 0.0f;
+#pragma unroll 4
+                    for (int j = 0; j < D / 8; ++j) {
+                        const uint4 v = vrow[j];
+                        const float4 qa = qrow[2 * j], qb = qrow[2 * j + 1];
+                        const float2 v0 = __half22float2(*reinterpret_cast<const __half2 *>(&v.x));
+                        const float2 v1 = __half22float2(*reinterpret_cast<const __half2 *>(&v.y));
+                        const float2 v2 = __half22float2(*reinterpret_cast<const __half2 *>(&v.z));
+                        const float2 v3 = __half22float2(*reinterpret_cast<const __half2 *>(&v.w));
+                        d0 = fmaf(qa.x, v0.x, d0);
+                        d1 = fmaf(qa.y, v0.y, d1);
+                        d0 = fmaf(qa.z, v1.x, d0);
+                        d1 = fmaf(qa.w, v1.y, d1);
+                        d0 = fmaf(qb.x, v2.x, d0);
+                        d1 = fmaf(qb.y, v2.y, d1);
+                        d0 = fmaf(qb.z, v3.x, d0);
+                        d1 = fmaf(qb.w, v3.y, d1);
+                    }
+                    dot = d0 + d1;
+                }
+                ws_split_store(b2, g, i, dot * WS_QSCALE);
+            }
+            fence_proxy_async_smem();
+            asm volatile("bar.sync 2, 64;" ::: "memory");
+            if (bt == 0) {
+                mbar_arrive(&bars.b2_full[vb]);
+                mbar_arrive(&bars.blk_empty[vb]);
+            }
+            if (first_of_head) {
+                first_of_head = false;
+                if ((head + 1) * a.bph < it1 && !build_w(head + 1, hidx + 1)) break;
+            }
+            jb += 1;
+            if (jb == a.bph) {
+                jb = 0;
+                head += 1;
+            }
+        }
+    }
+    else if (warp < 12) {
+        // ---------------------------------------------------------------- expanders (2 groups x 128 threads)
+        const int grp = (warp - 4) >> 2;
+        const int wt = ((warp - 4) & 3) * 32 + lane;   // token within the tile = tensor-memory lane
+        const uint32_t lane_base = static_cast<uint32_t>(32 * (warp & 3)) << 16;
+        uint32_t seq = 0, sbase = 0;
+        const uint32_t stages_per_block = (tiles + WS_TPS - 1) / WS_TPS;
+        bool alive = true;
+        for (int item = it0; item < it1 && alive; ++item, sbase += stages_per_block) {
+            for (int tile = 0; tile < tiles; ++tile, ++seq) {
+                if (static_cast<int>(seq & 1u) != grp) continue;
+                const uint32_t sseq = sbase + tile / WS_TPS;
+                const int stage = sseq % WS_STAGES, buf = seq & (WS_BUFS - 1);
+                if (!mbar_wait(&bars.st_full[stage], (sseq / WS_STAGES) & 1u, &abort_flag)) {
+                    alive = false;
+                    break;
+                }
+                const uint8_t *st = base + WS_OFF_STAGES + stage * WS_STAGE_BYTES;
+                const int rank = st_rank[stage];
+                const bool valid = tile * 128 + wt < n;
+                const int st_tok = (tile % WS_TPS) * 128 + wt;   // token within the stage
+                uint4 c0 = *reinterpret_cast<const uint4 *>(st + WS_ST_CODES + st_tok * 32);
+                uint4 c1 = *reinterpret_cast<const uint4 *>(st + WS_ST_CODES + st_tok * 32 + 16);
+                unsigned short rho_raw = *reinterpret_cast<const unsigned short *>(st + WS_ST_NORMS + st_tok * 2);
+                const uint8_t *pcol = st + WS_ST_P + (st_tok >> 8) * WS_ST_PBOX + (st_tok & 255) * 2;
+                uint32_t pw[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) pw[i] = 0u;
+#pragma unroll
+                for (int i = 0; i < WS_PMAX; ++i) {
+                    if (i < rank) {
+                        const uint32_t v = *reinterpret_cast<const unsigned short *>(pcol + i * 512);
+                        pw[i >> 1] |= v << (16 * (i & 1));
+                    }
+                }
+                {   // a stage is released by 128 arrivals per tile slot; the last tile of a short stage makes up the rest
+                    const int last_in_stage = min(tiles, (tile / WS_TPS + 1) * WS_TPS) - 1;
+                    const int arrivals = (tile == last_in_stage) ? 1 + (WS_TPS - 1 - (tile % WS_TPS)) : 1;
+                    for (int r = 0; r < arrivals; ++r) mbar_arrive(&bars.st_empty[stage]);
+                }
+                if (!valid) {   // rows past the end of the block were not copied: the stage holds stale bytes there
+                    c0 = make_uint4(0u, 0u, 0u, 0u);
+                    c1 = c0;
+                    rho_raw = 0;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) pw[i] = 0u;
+                }
+                const uint32_t u = (seq >> 2) & 1u;
+                if (!mbar_wait(&bars.a_empty[buf], u ^ 1u, &abort_flag) || !mbar_wait(&bars.d_empty[buf], u ^ 1u, &abort_flag)) {
+                    alive = false;
+                    break;
+                }
+                tc_fence_after_sync();
+                const uint32_t tb = tmem0 + lane_base + buf * WS_BUF_COLS;
+                {
+                    uint32_t av[32];
+                    const uint32_t w0[4] = {c0.x, c0.y, c0.z, c0.w}, w1[4] = {c1.x, c1.y, c1.z, c1.w};
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) ws_expand16(w0[q], a.lo_tab, a.hi_tab, &av[8 * q]);
+                    tmem_st32(tb, av);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) ws_expand16(w1[q], a.lo_tab, a.hi_tab, &av[8 * q]);
+                    tmem_st32(tb + 32, av);
+                }
+                tmem_st8(tb + WS_COL_P, pw);
+                {
+                    uint32_t rv[8];
+                    rv[0] = __float_as_uint(__half2float(__ushort_as_half(rho_raw)));
+#pragma unroll
+                    for (int i = 1; i < 8; ++i) rv[i] = 0u;
+                    tmem_st8(tb + WS_COL_RHO, rv);
+                }
+                tmem_st_wait();
+                tc_fence_before_sync();
+                mbar_arrive(&bars.a_full[buf]);
+            }
+        }
+    } else {
+        // ---------------------------------------------------------------- epilogue (128 threads)
+        const int wt = (warp & 3) * 32 + lane;
+        const uint32_t lane_base = static_cast<uint32_t>(32 * (warp & 3)) << 16;
+        const float f2 = a.scale * (1.0f / WS_QSCALE);
+        const size_t qstride = static_cast<size_t>(a.bph) * n;
+        uint32_t seq = 0;
+        bool alive = true;
+        int head = (it0 < it1) ? it0 / a.bph : 0, jb = it0 - head * a.bph;
+        for (int item = it0; item < it1 && alive; ++item) {
+            float *out_row = a.scores + (static_cast<size_t>(head) * a.G + a.g0) * qstride + static_cast<size_t>(jb) * n;
+            for (int tile = 0; tile < tiles; ++tile, ++seq) {
+                const int buf = seq & (WS_BUFS - 1);
+                if (!mbar_wait(&bars.d_full[buf], (seq >> 2) & 1u, &abort_flag)) {
+                    alive = false;
+                    break;
+                }
+                tc_fence_after_sync();
+                const uint32_t tb = tmem0 + lane_base + buf * WS_BUF_COLS;
+                uint32_t d1[16], d2[16], rv[8];
+                tmem_ld16(tb + WS_COL_D1, d1);
+                tmem_ld16(tb + WS_COL_D2, d2);
+                tmem_ld8(tb + WS_COL_RHO, rv);
+                tmem_ld_wait();
+                tc_fence_before_sync();
+                mbar_arrive(&bars.d_empty[buf]);
+                const int tok = tile * 128 + wt;
+                if (tok < n) {
+                    const float f1 = a.scale * __uint_as_float(rv[0]) * a.inv_code;
+#pragma unroll
+                    for (int g = 0; g < WS_NQ; ++g) {
+                        if (g < gcount) {
+                            const float code_part = __uint_as_float(d1[g]) + __uint_as_float(d1[WS_NQ + g]);
+                            const float low_part = __uint_as_float(d2[g]) + __uint_as_float(d2[WS_NQ + g]);
+                            out_row[static_cast<size_t>(g) * qstride + tok] = fmaf(f1, code_part, f2 * low_part);
+                        }
+                    }
+                }
+            }
+            jb += 1;
+            if (jb == a.bph) {
+                jb = 0;
+                head += 1;
+            }
+        }
+    }
+
+    __syncthreads();
+    if (abort_flag && tid == 0) atomicOr(a.err, TC_ERR_SCORES_WS_TIMEOUT);
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem0, WS_TMEM_COLS);
+    }
+}
+
+bool scores_ws_supported(const eosq_cache_t &cache, int bits, int n) {
+    auto aligned = [](const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; };
+    return bits == 2 && n >= 128 && (n % 8) == 0 && aligned(cache.codes) && aligned(cache.norms) && aligned(cache.P) && aligned(cache.V);
+}
+
+bool launch_scores_ws(const eosq_cache_t &cache, int64_t heads, int64_t bph, int64_t head_stride, int n, const Rotation &rot,
+                      const uint16_t (&table)[16], float kappa, const __half *q, int G, float scale, float *scores, int *err,
+                      int sm_count, cudaStream_t s) {
+    static bool configured = false;
+    if (!configured) {
+        if (cudaFuncSetAttribute(scores_ws_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(WS_SMEM_BYTES)) != cudaSuccess)
+            return false;
+        configured = true;
+    }
+    if (heads * bph > 0x7fffffff || head_stride > 0x7fffffff) return false;
+    WsArgs a;
+    a.cache = cache;
+    a.bph = static_cast<int>(bph);
+    a.head_stride = static_cast<int>(head_stride);
+    a.heads = static_cast<int>(heads);
+    a.n = n;
+    a.G = G;
+    a.scale = scale;
+    a.inv_code = 1.0f / (kappa * WS_QSCALE);
+    a.lo_tab = 0u;
+    a.hi_tab = 0u;
+    for (int k = 0; k < 4; ++k) {
+        a.lo_tab |= static_cast<uint32_t>(table[k] & 0xFFu) << (8 * k);
+        a.hi_tab |= static_cast<uint32_t>(table[k] >> 8) << (8 * k);
+    }
+    a.pi_t = rot.pi_t;
+    a.q = q;
+    a.scores = scores;
+    a.err = err;
+    const int grid = static_cast<int>(std::min<int64_t>(heads * bph, sm_count));
+    const int64_t nb_total = (heads - 1) * head_stride + bph;
+    CUtensorMap m4, m8, m12;
+    if (!make_factor_tensor_map(cache.P, nb_total, n, 4, &m4) || !make_factor_tensor_map(cache.P, nb_total, n, 8, &m8) ||
+        !make_factor_tensor_map(cache.P, nb_total, n, 12, &m12))
+        return false;
+    for (int g0 = 0; g0 < G; g0 += WS_NQ) {
+        a.g0 = g0;
+        scores_ws_kernel<<<grid, WS_THREADS, WS_SMEM_BYTES, s>>>(a, m4, m8, m12);
+    }
+    return true;
+}
+
+}  // namespace eosq

@@ -51,6 +51,20 @@ bool make_block_tensor_map(const void *blocks, int64_t nb, int n, CUtensorMap *o
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Unswizzled tensor map over the stored left factors P [B][RMAX][n] fp16 with boxes of `rows`
+// factor rows x 256 tokens (a box lands in shared memory as `rows` lines of 512 bytes).
+bool make_factor_tensor_map(const void *P, int64_t nb, int n, int rows, CUtensorMap *out) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {static_cast<cuuint64_t>(n), static_cast<cuuint64_t>(RMAX), static_cast<cuuint64_t>(nb)};
+    const cuuint64_t strides[2] = {static_cast<cuuint64_t>(n) * 2, static_cast<cuuint64_t>(n) * RMAX * 2};
+    const cuuint32_t box[3] = {256, static_cast<cuuint32_t>(rows), 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void *>(P), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // ------------------------------------------------------------------------------------------
 // Gram matrix.  Persistent CTAs, 320 threads: warp 0 loads token tiles by TMA into a ring of
 // stages, warp 1 issues the MMAs, warps 2-9 add finished partial sums into fp64 registers.
