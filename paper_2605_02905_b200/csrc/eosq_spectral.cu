@@ -564,18 +564,24 @@ __global__ void __launch_bounds__(256) spectral_kernel(int n, Workspace ws, eosq
             y0[m] = yv[(lane + 32 * m) * LU_LANES + i0];
             y1[m] = two ? yv[(lane + 32 * m) * LU_LANES + i1] : 0.0;
         }
+        // the reflector of the next step is fetched while the current one is applied
+        double nx[4];
+#pragma unroll
+        for (int m = 0; m < 4; ++m) nx[m] = R[static_cast<size_t>(D - 3) * D + lane + 32 * m];
         for (int k = D - 3; k >= 0; --k) {
             const double t = tt[k];
-            if (t == 0.0) continue;
-            const double *row = R + static_cast<size_t>(k) * D;
             double vv[4], dot0 = 0.0, dot1 = 0.0;
 #pragma unroll
             for (int m = 0; m < 4; ++m) {
-                const int j = lane + 32 * m;
-                vv[m] = row[j];
+                vv[m] = nx[m];
                 dot0 += vv[m] * y0[m];
                 dot1 += vv[m] * y1[m];
             }
+            if (k > 0) {
+#pragma unroll
+                for (int m = 0; m < 4; ++m) nx[m] = R[static_cast<size_t>(k - 1) * D + lane + 32 * m];
+            }
+            if (t == 0.0) continue;
             dot0 = t * warp_sum(dot0);
             dot1 = t * warp_sum(dot1);
 #pragma unroll
