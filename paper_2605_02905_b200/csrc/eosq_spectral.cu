@@ -474,7 +474,10 @@ __global__ void __launch_bounds__(256) spectral_kernel(int n, Workspace ws, eosq
         }
 
         // Kept eigenvectors of the tridiagonal matrix: (T - mu I) = P L U with partial pivoting,
-        // three steps of inverse iteration.  Lane i of warp 0 owns vector i (column i of the arrays).
+        // two steps of inverse iteration (the kept eigenvalues are separated from their
+        // neighbours by far more than their error, so each step gains many digits).  Lane i of
+        // warp 0 owns vector i (column i of the arrays).  The iterate is left unnormalised: it can
+        // grow by at most 1 / floor_piv per step, and the back-transformation normalises at the end.
         if (warp == 0 && lane < rank) {
             const int c = lane;
             const double mu = lam[c];
@@ -485,40 +488,40 @@ __global__ void __launch_bounds__(256) spectral_kernel(int n, Workspace ws, eosq
                 const double l = ee[i];
                 const double d_next = dd[i + 1] - mu;
                 const double u_next = (i + 1 < D - 1) ? ee[i + 1] : 0.0;
+                const bool keep = fabs(d_i) >= fabs(l);
+                double pv = keep ? d_i : l;   // the pivot; its reciprocal serves the elimination and the back substitution
+                if (!(fabs(pv) >= floor_piv)) pv = (pv < 0.0) ? -floor_piv : floor_piv;
+                const double inv = 1.0 / pv;
                 double fact, nd, nu;
-                if (fabs(d_i) >= fabs(l)) {
-                    fact = (d_i != 0.0) ? l / d_i : 0.0;
-                    lu_d[i * LU_LANES + c] = d_i;
+                if (keep) {
+                    fact = l * inv;
                     lu_u[i * LU_LANES + c] = u_i;
                     lu_u2[i * LU_LANES + c] = 0.0;
                     nd = d_next - fact * u_i;
                     nu = u_next;
                 } else {
-                    fact = d_i / l;
-                    lu_d[i * LU_LANES + c] = l;
+                    fact = d_i * inv;
                     lu_u[i * LU_LANES + c] = d_next;
                     lu_u2[i * LU_LANES + c] = u_next;
                     nd = u_i - fact * d_next;
                     nu = -fact * u_next;
                     piv[i >> 5] |= 1u << (i & 31);
                 }
+                lu_d[i * LU_LANES + c] = inv;
                 lu_l[i * LU_LANES + c] = fact;
                 d_i = nd;
                 u_i = nu;
             }
-            lu_d[(D - 1) * LU_LANES + c] = d_i;
+            if (!(fabs(d_i) >= floor_piv)) d_i = (d_i < 0.0) ? -floor_piv : floor_piv;
+            lu_d[(D - 1) * LU_LANES + c] = 1.0 / d_i;
             lu_u[(D - 1) * LU_LANES + c] = 0.0;
             lu_u2[(D - 1) * LU_LANES + c] = 0.0;
-            for (int i = 0; i < D; ++i) {
-                double x = lu_d[i * LU_LANES + c];
-                if (!(fabs(x) >= floor_piv)) x = (x < 0.0) ? -floor_piv : floor_piv;
-                lu_d[i * LU_LANES + c] = 1.0 / x;
-            }
             for (int i = 0; i < D; ++i) {
                 const double f = (i + 1) * 0.6180339887498949;
                 yv[i * LU_LANES + c] = 0.5 + (f - floor(f));
             }
-            for (int it = 0; it < 3; ++it) {
+            double ss = 0.0;
+            for (int it = 0; it < 2; ++it) {
                 double carry = yv[c];
                 for (int i = 0; i < D - 1; ++i) {  // forward: apply the row interchanges and L^-1
                     const double next = yv[(i + 1) * LU_LANES + c];
@@ -533,7 +536,8 @@ __global__ void __launch_bounds__(256) spectral_kernel(int n, Workspace ws, eosq
                 }
                 double x1 = carry * lu_d[(D - 1) * LU_LANES + c];  // backward: U^-1
                 yv[(D - 1) * LU_LANES + c] = x1;
-                double x2 = 0.0, ss = x1 * x1;
+                double x2 = 0.0;
+                ss = x1 * x1;
                 for (int i = D - 2; i >= 0; --i) {
                     const double x = (yv[i * LU_LANES + c] - lu_u[i * LU_LANES + c] * x1 - lu_u2[i * LU_LANES + c] * x2) *
                                      lu_d[i * LU_LANES + c];
@@ -542,12 +546,8 @@ __global__ void __launch_bounds__(256) spectral_kernel(int n, Workspace ws, eosq
                     x2 = x1;
                     x1 = x;
                 }
-                // normalise in two steps so that the squares cannot overflow
-                const double big = sqrt(ss);
-                const double inv = (big > 0.0 && big < 1e300) ? 1.0 / big : 1.0;
-                if (!(big > 0.0 && big < 1e300)) atomicOr(&s_flags, EOSQ_BLOCK_NOT_CONVERGED);
-                for (int i = 0; i < D; ++i) yv[i * LU_LANES + c] *= inv;
             }
+            if (!(ss > 0.0 && ss < 1e300)) atomicOr(&s_flags, EOSQ_BLOCK_NOT_CONVERGED);
         }
     }
     __syncthreads();
