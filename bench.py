@@ -245,8 +245,14 @@ def run_library(args):
     dom_ms_per_launch = stage[dominant][0] / max(dom_launches, 1)
     blocks_per_launch = B * args.steps / max(dom_launches, 1)
     achieved = units * blocks_per_launch / (dom_ms_per_launch * 1e-3)
+    # DRAM bytes per block from the committed ncu section capture (profiles/sections_per_kernel_*.txt),
+    # scaled to the blocks of one launch; None for kernels changed since that capture
+    ncu_traffic_per_block = {"tridiag": 97.4e6 / 592, "gram": 186e6 / 592, "quant": 179e6 / 592, "eigvals": 1.2e6 / 592}
+    traffic = ncu_traffic_per_block.get(dominant)
     roofline = {"kernel": dominant, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit,
-                "frac": achieved / peak, "traffic": None, "peak_source": peaks["source"],
+                "frac": achieved / peak, "traffic": (traffic * blocks_per_launch if traffic else None),
+                "traffic_note": "dram__bytes (read+write) of one 592-block launch under ncu, scaled by blocks per launch",
+                "peak_source": peaks["source"],
                 "ms_per_launch": dom_ms_per_launch, "launches": dom_launches}
     # whole encode against the task's roofline: slower of bytes at HBM peak and Gram+rotation flops at tensor peak
     t_hbm = (in_bytes + B * out_bytes_per_block) / (peaks["hbm_gbs"] * 1e9)
