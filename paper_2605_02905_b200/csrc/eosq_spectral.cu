@@ -252,7 +252,7 @@ __global__ void __launch_bounds__(TD_THREADS, 1) tridiag_kernel(double *__restri
 // the number of sign changes in p_0 .. p_d is the number of eigenvalues below x.  One thread per
 // eigenvalue.  A first pass counts at 128 points spaced geometrically below the Gershgorin bound
 // (the spectrum of a Gram matrix spans many decades), which brackets every eigenvalue to 18 %;
-// bisection then runs until the bracket is below 1e-10 relative (2e-15 of the matrix scale for the
+// bisection then runs until the bracket is below 1e-8 relative (2e-15 of the matrix scale for the
 // smallest ones).
 // ------------------------------------------------------------------------------------------
 constexpr double EV_E2_FLOOR = 1e-60;   // keeps the recurrence alive across an exactly decoupled entry
@@ -364,7 +364,7 @@ __global__ void __launch_bounds__(D) eigvals_kernel(const double *__restrict__ d
     if (t == D - 1) lo = hi;   // cannot happen (every eigenvalue is below the last point); keeps the bracket sane
     for (int it = 0; it < EV_MAX_BISECT; ++it) {
         const double mid = 0.5 * (lo + hi);
-        const bool done = (hi - lo) <= fmax(2e-15, 1e-10 * fabs(mid));
+        const bool done = (hi - lo) <= fmax(2e-15, 1e-8 * fabs(mid));
         if (__all_sync(0xffffffffu, done)) break;
         if (sturm_count(sde, mid) > target) hi = mid;
         else lo = mid;
