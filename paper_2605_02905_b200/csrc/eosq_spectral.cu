@@ -34,15 +34,16 @@ struct TdShared {
     double up[2][TD_PLEN];     // u, permuted (16-byte aligned by the struct's placement)
     double pp[2][TD_PLEN];     // p, permuted
     double wsum[2][8];
-    double sgam[2];
+    double sspart[2][16];      // partial sums of squares of the published row, one per holder thread
     double dg[D], of[D], ta[D];
 };
 
-// The sixteen threads that hold row r (slot AR = r / 16 of their tiles) publish its tail as the
-// reflector of step r into buffer `nxt`.  Only slots b >= AR can hold columns j > r.
+// The sixteen threads that hold row r (slot AR = r / 16 of their tiles) publish its raw tail
+// x = A[r][r+1..] into buffer `nxt`, together with their partial sums of squares of x[r+2..].  The
+// norm, beta and gamma of the reflector are worked out by every thread after the next barrier, in
+// the shadow of the matrix-vector product, instead of by these sixteen while the CTA waits.
 template <int AR>
-__device__ __forceinline__ void td_publish(const double (&A)[8][8], int r, int nxt, int tc, int lane, TdShared &sh) {
-    const unsigned mask = 0xFFFFu << (lane & 16);
+__device__ __forceinline__ void td_publish(const double (&A)[8][8], int r, int nxt, int tc, TdShared &sh) {
     double x[8];
     double ss0 = 0.0, ss1 = 0.0;
 #pragma unroll
@@ -64,25 +65,7 @@ __device__ __forceinline__ void td_publish(const double (&A)[8][8], int r, int n
     dst[1] = make_double2(x[2], x[3]);
     dst[2] = make_double2(x[4], x[5]);
     dst[3] = make_double2(x[6], x[7]);
-    double ss = ss0 + ss1;
-#pragma unroll
-    for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(mask, ss, o);
-    __syncwarp(mask);
-    const double alpha = sh.up[nxt][td_pos(r + 1)];
-    double beta = alpha, gamma = 0.0;
-    if (ss > 0.0) {
-        const double s2 = fma(alpha, alpha, ss);
-        const double nrm = s2 * rsqrt(s2);
-        beta = (alpha >= 0.0) ? -nrm : nrm;
-        gamma = 1.0 / fma(fabs(alpha), nrm, s2);   // 1 / (beta (beta - alpha))
-    }
-    __syncwarp(mask);
-    if (tc == 0) {
-        sh.up[nxt][td_pos(r + 1)] = alpha - beta;
-        sh.sgam[nxt] = gamma;
-        sh.of[r] = beta;
-        sh.ta[r] = gamma;
-    }
+    sh.sspart[nxt][tc] = ss0 + ss1;
 }
 
 // One step k with (k + 1) / 16 == K0: tile slots below K0 hold only finished rows and columns and
@@ -92,9 +75,29 @@ __device__ __forceinline__ void td_step(double (&A)[8][8], int k, int tid, TdSha
     const int lane = tid & 31, warp = tid >> 5, tr = tid >> 4, tc = tid & 15;
     __syncthreads();
     const int cur = k & 1;
-    const double gamma = sh.sgam[cur];
-    if (tid < D) refl[k * D + tid] = (tid > k) ? sh.up[cur][td_pos(tid)] : 0.0;
+    // reflector scalars from the published row: u = x - beta e_{k+1}, H = I - gamma u u^T
+    double ss;
+    {
+        const double2 *sp = reinterpret_cast<const double2 *>(sh.sspart[cur]);
+        const double2 s0 = sp[0], s1 = sp[1], s2 = sp[2], s3 = sp[3], s4 = sp[4], s5 = sp[5], s6 = sp[6], s7 = sp[7];
+        ss = (((s0.x + s0.y) + (s1.x + s1.y)) + ((s2.x + s2.y) + (s3.x + s3.y))) +
+             (((s4.x + s4.y) + (s5.x + s5.y)) + ((s6.x + s6.y) + (s7.x + s7.y)));
+    }
+    const double alpha = sh.up[cur][td_pos(k + 1)];
+    double beta = alpha, gamma = 0.0;
+    if (ss > 0.0) {
+        const double sq = fma(alpha, alpha, ss);
+        const double nrm = sq * rsqrt(sq);
+        beta = (alpha >= 0.0) ? -nrm : nrm;
+        gamma = 1.0 / fma(fabs(alpha), nrm, sq);   // 1 / (beta (beta - alpha))
+    }
+    if (tid < D) refl[k * D + tid] = (tid > k) ? sh.up[cur][td_pos(tid)] - ((tid == k + 1) ? beta : 0.0) : 0.0;
+    if (tid == 0) {
+        sh.of[k] = beta;
+        sh.ta[k] = gamma;
+    }
     const bool owner = (tr == ((k + 1) & 15)) && (k + 1 < D - 2);
+    const bool col_holder = tc == ((k + 1) & 15), row_holder = tr == ((k + 1) & 15);   // of index k + 1 (tile slot K0)
     if (gamma != 0.0) {   // uniform over the CTA
         double uj[8], ui[8], acc[8];
         {
@@ -109,7 +112,8 @@ __device__ __forceinline__ void td_step(double (&A)[8][8], int k, int tid, TdSha
                 ui[2 * q + 1] = w.y;
             }
         }
-        double tloc = 0.0;
+        // A x with the raw row (independent of beta, so it overlaps the square root and the division
+        // above), then the - beta A e_{k+1} term from the threads that hold column k + 1
 #pragma unroll
         for (int a = 0; a < 8; ++a) {
             acc[a] = 0.0;
@@ -121,8 +125,15 @@ __device__ __forceinline__ void td_step(double (&A)[8][8], int k, int tid, TdSha
                     else s0 = fma(A[a][b], uj[b], s0);
                 }
                 acc[a] = s0 + s1;
-                tloc = fma(ui[a], acc[a], tloc);
             }
+        }
+        double tloc = 0.0;
+        if (col_holder) uj[K0] -= beta;
+        if (row_holder) ui[K0] -= beta;
+#pragma unroll
+        for (int a = K0; a < 8; ++a) {
+            if (col_holder) acc[a] = fma(-beta, A[a][K0], acc[a]);
+            tloc = fma(ui[a], acc[a], tloc);
         }
         // sum the partial rows over the sixteen column groups: each stage keeps half of the rows
         const bool h8 = tc & 8, h4 = tc & 4, h2 = tc & 2;
@@ -170,7 +181,7 @@ __device__ __forceinline__ void td_step(double (&A)[8][8], int k, int tid, TdSha
         if (owner) {
 #pragma unroll
             for (int b = K0; b < 8; ++b) A[K0][b] = fma(-ui[K0], pj[b], fma(-si[K0], uj[b], A[K0][b]));
-            td_publish<K0>(A, k + 1, cur ^ 1, tc, lane, sh);
+            td_publish<K0>(A, k + 1, cur ^ 1, tc, sh);
         }
 #pragma unroll
         for (int a = K0; a < 8; ++a) {
@@ -180,7 +191,7 @@ __device__ __forceinline__ void td_step(double (&A)[8][8], int k, int tid, TdSha
             }
         }
     } else if (owner) {
-        td_publish<K0>(A, k + 1, cur ^ 1, tc, lane, sh);
+        td_publish<K0>(A, k + 1, cur ^ 1, tc, sh);
     }
 }
 
@@ -214,7 +225,7 @@ __global__ void __launch_bounds__(TD_THREADS, 1) tridiag_kernel(double *__restri
         for (int b = 0; b < 8; ++b) A[a][b] = td_refl[(tr + 16 * a) * D + tc + 16 * b];
     __syncthreads();
 
-    if (tr == 0) td_publish<0>(A, 0, 0, tc, lane, sh);
+    if (tr == 0) td_publish<0>(A, 0, 0, tc, sh);
 #pragma unroll 1
     for (int k = 0; k < D - 2; ++k) {
         switch ((k + 1) >> 4) {
