@@ -345,10 +345,22 @@ __global__ void __launch_bounds__(QT_THREADS, 2) quant_tc_kernel(const __grid_co
 #pragma unroll
             for (int i = 0; i < 8; ++i) w[i] = 0.0f;
             if (8 * half < rank) {
-                for (int j = 0; j < D; ++j) {
-                    const float pv = pi_t[j * D + c];
+#pragma unroll 1
+                for (int j0 = 0; j0 < D; j0 += 32) {
+                    float pv[32];
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) w[i] = fmaf(pv, Vc[(8 * half + i) * D + j], w[i]);
+                    for (int jj = 0; jj < 32; ++jj) pv[jj] = __ldg(pi_t + (j0 + jj) * D + c);   // 32 loads in flight
+#pragma unroll
+                    for (int jj = 0; jj < 32; jj += 4) {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {   // one 16-byte broadcast load feeds four multiply-adds
+                            const float4 vv = *reinterpret_cast<const float4 *>(Vc + (8 * half + i) * D + j0 + jj);
+                            w[i] = fmaf(pv[jj], vv.x, w[i]);
+                            w[i] = fmaf(pv[jj + 1], vv.y, w[i]);
+                            w[i] = fmaf(pv[jj + 2], vv.z, w[i]);
+                            w[i] = fmaf(pv[jj + 3], vv.w, w[i]);
+                        }
+                    }
                 }
             }
 #pragma unroll
@@ -463,21 +475,44 @@ __global__ void __launch_bounds__(QT_THREADS, 2) quant_tc_kernel(const __grid_co
             __syncthreads();   // both halves of every row are summed; every warp has read its accumulator part
             const float tot = ss_part[0][row] + ss_part[1][row];
             const float rho = sqrtf(tot);
-            const float inv = (rho > 0.0f) ? 1.0f / rho : 0.0f;
+            // thresholds scaled by the norm: y > thr rho decides as y / rho > thr does (a zero row keeps
+            // the plain thresholds, so that it gets the code of z = 0)
+            float ts[NTHR];
+#pragma unroll
+            for (int k = 0; k < NTHR; ++k) ts[k] = (rho > 0.0f) ? thr[k] * rho : thr[k];
             unsigned long long wv[BITS];
+            if (BITS == 3) {
 #pragma unroll
-            for (int k = 0; k < BITS; ++k) wv[k] = 0ull;
+                for (int k = 0; k < BITS; ++k) wv[k] = 0ull;
 #pragma unroll
-            for (int c = 0; c < 64; ++c) {
-                const float z = y[c] * inv;
-                unsigned code = 0u;
+                for (int c = 0; c < 64; ++c) {
+                    unsigned code = 0u;
 #pragma unroll
-                for (int k = 0; k < NTHR; ++k) code += (thr[k] < z) ? 1u : 0u;
-                constexpr int dummy = 0;
-                (void)dummy;
-                const int pos = c * BITS;
-                wv[pos >> 6] |= static_cast<unsigned long long>(code) << (pos & 63);
-                if ((pos & 63) + BITS > 64) wv[(pos >> 6) + 1] |= static_cast<unsigned long long>(code) >> (64 - (pos & 63));
+                    for (int k = 0; k < NTHR; ++k) code += (ts[k] < y[c]) ? 1u : 0u;
+                    const int pos = c * BITS;
+                    wv[pos >> 6] |= static_cast<unsigned long long>(code) << (pos & 63);
+                    if ((pos & 63) + BITS > 64) wv[(pos >> 6) + 1] |= static_cast<unsigned long long>(code) >> (64 - (pos & 63));
+                }
+            } else {
+                constexpr int CPW = 32 / BITS;   // codes per 32-bit word, filled from the top code down
+#pragma unroll
+                for (int k = 0; k < BITS; ++k) {
+                    uint32_t w2[2];
+#pragma unroll
+                    for (int hw = 0; hw < 2; ++hw) {
+                        uint32_t w = 0u;
+#pragma unroll
+                        for (int e = CPW - 1; e >= 0; --e) {
+                            const float v = y[(2 * k + hw) * CPW + e];
+                            uint32_t code = 0u;
+#pragma unroll
+                            for (int t = 0; t < NTHR; ++t) code += (ts[t] < v) ? 1u : 0u;
+                            w = w * (1u << BITS) + code;
+                        }
+                        w2[hw] = w;
+                    }
+                    wv[k] = static_cast<unsigned long long>(w2[0]) | (static_cast<unsigned long long>(w2[1]) << 32);
+                }
             }
             if (tok < n) {
                 unsigned long long *dst = reinterpret_cast<unsigned long long *>(
