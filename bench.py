@@ -233,7 +233,9 @@ def run_library(args):
     algo = {
         # stage: (bound, algorithmic units per block, peak, unit)
         "gram": ("tensor", 2.0 * n * d * d / 1e12, peaks["bf16_tflops_sustained"], "TFLOP/s"),
-        "tridiag": ("alu", (4.0 / 3.0) * d ** 3 / 1e12, FP64_PEAK_TFLOPS, "TFLOP/s"),
+        # Householder tridiagonalisation: 4/3 m^3 flops for order m; the head kernel takes d -> d/2, the tail the rest
+        "tridiag_head": ("alu", (4.0 / 3.0) * (d ** 3 - (d // 2) ** 3) / 1e12, FP64_PEAK_TFLOPS, "TFLOP/s"),
+        "tridiag_tail": ("alu", (4.0 / 3.0) * (d // 2) ** 3 / 1e12, FP64_PEAK_TFLOPS, "TFLOP/s"),
         "eigvals": ("alu", 32 * d * d * 6.0 / 1e12, FP64_PEAK_TFLOPS, "TFLOP/s"),   # ~32 Sturm counts x d steps x 3 fp64 ops per eigenvalue
         "spectral": ("alu", (4.0 * d * d * max(mean_rank, 1.0)) / 1e12, FP64_PEAK_TFLOPS, "TFLOP/s"),
         "quant": ("hbm", (n * d * 2 + out_bytes_per_block) / 1e9, peaks["hbm_gbs"], "GB/s"),
@@ -247,7 +249,7 @@ def run_library(args):
     achieved = units * blocks_per_launch / (dom_ms_per_launch * 1e-3)
     # DRAM bytes per block from the committed ncu section capture (profiles/sections_per_kernel_*.txt),
     # scaled to the blocks of one launch; None for kernels changed since that capture
-    ncu_traffic_per_block = {"tridiag": 97.4e6 / 592, "gram": 186e6 / 592, "quant": 179e6 / 592, "eigvals": 1.2e6 / 592}
+    ncu_traffic_per_block = {"gram": 186e6 / 592}
     traffic = ncu_traffic_per_block.get(dominant)
     roofline = {"kernel": dominant, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit,
                 "frac": achieved / peak, "traffic": (traffic * blocks_per_launch if traffic else None),

@@ -205,10 +205,11 @@ int64_t eosq_launch_count(const eosq_ctx *ctx);
  * CUDA events on the launching stream.  eosq_profile_read synchronises those events, adds their
  * elapsed milliseconds into ms[EOSQ_NUM_STAGES] and their launch counts into
  * launches[EOSQ_NUM_STAGES] (host arrays, overwritten), and clears the record.
- * Stage order: Gram, tridiagonalisation, eigenvalues, spectrum + shrinkage + eigenvectors,
+ * Stage order: Gram, tridiagonalisation (first 64 steps), tridiagonalisation (trailing 64 x 64
+ * matrix), eigenvalues, spectrum + shrinkage + eigenvectors,
  * residual/rotate/quantise/pack, decode, scores.
  */
-#define EOSQ_NUM_STAGES 8
+#define EOSQ_NUM_STAGES 9
 int eosq_profile_enable(eosq_ctx *ctx, int on);
 int eosq_profile_read(eosq_ctx *ctx, float *ms, int64_t *launches);
 

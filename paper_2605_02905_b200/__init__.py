@@ -29,7 +29,7 @@ EXPORTS = [
     "eosq_check_status", "eosq_launch_count", "eosq_profile_enable", "eosq_profile_read",
     "eosq_encode_static", "eosq_encode_static_max_blocks",
 ]
-STAGES = ["gram", "tridiag", "eigvals", "spectral", "quant", "decode", "scores", "other"]
+STAGES = ["gram", "tridiag_head", "tridiag_tail", "eigvals", "spectral", "quant", "decode", "scores", "other"]
 
 
 class EosqError(RuntimeError):
@@ -172,10 +172,10 @@ class Context:
 
     def profile_read(self) -> dict:
         """{stage: (milliseconds, launches)} accumulated since the last read (synchronises)."""
-        ms = (ctypes.c_float * 8)()
-        cnt = (ctypes.c_int64 * 8)()
+        ms = (ctypes.c_float * len(STAGES))()
+        cnt = (ctypes.c_int64 * len(STAGES))()
         _check(lib().eosq_profile_read(self._h, ms, cnt), "eosq_profile_read", self)
-        return {STAGES[i]: (float(ms[i]), int(cnt[i])) for i in range(8)}
+        return {STAGES[i]: (float(ms[i]), int(cnt[i])) for i in range(len(STAGES))}
 
 
 @dataclass

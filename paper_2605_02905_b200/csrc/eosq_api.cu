@@ -129,14 +129,17 @@ int eosq::encode_chunk(eosq_ctx *ctx, const void *blocks, int in_dtype, int64_t 
     } else {
         run_stage(ctx, ST_GRAM, s, [&] { launch_gram_plain(chunk_in, in_dtype, nb, n, ws.gram, nullptr, nullptr, s); });
     }
-    run_stage(ctx, ST_TRIDIAG, s, [&] { launch_tridiag(nb, ws, nullptr, nullptr, s); });
+    for (int part = 0; part < TRIDIAG_PARTS; ++part)
+        run_stage(ctx, part + 1 < TRIDIAG_PARTS ? ST_TRIDIAG_HEAD : ST_TRIDIAG_TAIL, s, [&] { launch_tridiag(part, nb, ws, nullptr, nullptr, s); });
     run_stage(ctx, ST_EIGVALS, s, [&] { launch_eigvals(nb, ws, nullptr, nullptr, s); });
     if (in_dtype == EOSQ_F16) {
         // second pass, exact Gram matrix, for the blocks the tensor-core one cannot resolve
         if (record_cuda(ctx, cudaMemsetAsync(ws.redo_count, 0, sizeof(int), s), "cudaMemsetAsync(redo count)")) return EOSQ_ERR_CUDA;
         run_stage(ctx, ST_OTHER, s, [&] { launch_mark_redo(nb, ws, s); });
         run_stage(ctx, ST_GRAM, s, [&] { launch_gram_plain(chunk_in, in_dtype, nb, n, ws.gram, ws.redo_list, ws.redo_count, s); });
-        run_stage(ctx, ST_TRIDIAG, s, [&] { launch_tridiag(nb, ws, ws.redo_list, ws.redo_count, s); });
+        for (int part = 0; part < TRIDIAG_PARTS; ++part)
+            run_stage(ctx, part + 1 < TRIDIAG_PARTS ? ST_TRIDIAG_HEAD : ST_TRIDIAG_TAIL, s,
+                      [&] { launch_tridiag(part, nb, ws, ws.redo_list, ws.redo_count, s); });
         run_stage(ctx, ST_EIGVALS, s, [&] { launch_eigvals(nb, ws, ws.redo_list, ws.redo_count, s); });
     }
     run_stage(ctx, ST_SPECTRAL, s, [&] { launch_spectral(nb, n, ws, o, 0, s); });

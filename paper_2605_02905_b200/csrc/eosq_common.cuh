@@ -83,7 +83,7 @@ inline size_t carve(void *base, int64_t cap, Workspace *ws) {
 
 }  // namespace eosq
 
-enum Stage { ST_GRAM = 0, ST_TRIDIAG, ST_EIGVALS, ST_SPECTRAL, ST_QUANT, ST_DECODE, ST_SCORES, ST_OTHER };
+enum Stage { ST_GRAM = 0, ST_TRIDIAG_HEAD, ST_TRIDIAG_TAIL, ST_EIGVALS, ST_SPECTRAL, ST_QUANT, ST_DECODE, ST_SCORES, ST_OTHER };
 
 struct eosq_ctx {
     struct Timed {
@@ -120,7 +120,8 @@ void launch_gram_plain(const void *blocks, int in_dtype, int64_t nb, int n, doub
 bool launch_gram_tc(const void *blocks_all, int64_t nb_all, int64_t block0, int64_t nb, int n, double *gram, int *err,
                     int sm_count, cudaStream_t s);
 // Householder tridiagonalisation of each Gram matrix (in place: reflectors overwrite it).
-void launch_tridiag(int64_t nb, const Workspace &ws, const int *list, const int *count, cudaStream_t s);
+constexpr int TRIDIAG_PARTS = 3;
+void launch_tridiag(int part, int64_t nb, const Workspace &ws, const int *list, const int *count, cudaStream_t s);
 // All eigenvalues of each tridiagonal matrix by Sturm bisection.
 void launch_eigvals(int64_t nb, const Workspace &ws, const int *list, const int *count, cudaStream_t s);
 // Clears the redo list / appends every block whose eigenvalue range exceeds 1 / REDO_RATIO.

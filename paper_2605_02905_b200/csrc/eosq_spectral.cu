@@ -10,40 +10,48 @@
 namespace eosq {
 
 // ------------------------------------------------------------------------------------------
-// Householder tridiagonalisation, one CTA (256 threads) per matrix, the matrix resident in
-// registers as 8 x 8 cyclic tiles: thread (tr, tc) = (tid / 16, tid % 16) holds
-// A[tr + 16 a][tc + 16 b], a, b < 8, so every thread keeps an equal share of the shrinking
-// trailing matrix, and a vector entry fetched from shared memory feeds eight multiply-adds.
+// Householder tridiagonalisation with the matrix resident in registers as 8 x 8 cyclic tiles on a
+// G x G thread grid: thread (tr, tc) = (tid / G, tid % G) holds A[tr + G a][tc + G b], a, b < 8,
+// so every thread keeps an equal share of the shrinking trailing matrix, and a vector entry
+// fetched from shared memory feeds eight multiply-adds.
 //
-// Step k reflects with H = I - gamma u u^T, u = (0, .., 0, alpha - beta, A[k][k+2], .., A[k][d-1]),
+// Step k reflects with H = I - gamma u u^T, u = (0, .., 0, alpha - beta, A[k][k+2], .., A[k][N-1]),
 // alpha = A[k][k+1], beta = -sign(alpha) ||A[k][k+1..]||, gamma = 1 / (beta (beta - alpha)):
 //     p = gamma A u,  2K = gamma (u.p),  A <- A - u p^T - (p - 2K u) u^T.
 // u and p travel through shared memory (double buffered by the parity of k, two block-wide
 // barriers per step) in a permuted order that makes a thread's eight columns contiguous.
-// Reflectors and the tridiagonal entries are collected in shared memory and written out at the
-// end: row k of the matrix in global memory receives u, tau[k] receives gamma.
+//
+// Every step is a chain of dependent latencies (two barriers, a square root and a division, a
+// butterfly reduction), so one matrix cannot fill an SM.  The work is therefore split in two
+// kernels.  The head (G = 16, 256 threads, one CTA per SM) takes the 128 x 128 matrix through its
+// first 64 steps and leaves the 64 x 64 trailing matrix in the lower left quadrant of the matrix
+// in global memory, which no reflector uses.  The tail (G = 8, 64 threads) finishes that trailing
+// matrix with four CTAs per SM, whose latency chains overlap.  Row k of the matrix in global
+// memory receives u of step k, tau[k] receives gamma.
 // ------------------------------------------------------------------------------------------
-constexpr int TD_THREADS = 256;
 constexpr int TD_PSTRIDE = 10;   // doubles per column group in the permuted vectors (8 used, 2 pad)
-constexpr int TD_PLEN = 16 * TD_PSTRIDE;
 
-__device__ __forceinline__ int td_pos(int j) { return (j & 15) * TD_PSTRIDE + (j >> 4); }
+template <int G>
+__device__ __forceinline__ int td_pos(int j) {
+    return (j & (G - 1)) * TD_PSTRIDE + (j / G);
+}
 
-// Shared-memory state of one tridiagonalisation.
+// Shared-memory state of one tridiagonalisation of order 8 G.
+template <int G>
 struct TdShared {
-    double up[2][TD_PLEN];     // u, permuted (16-byte aligned by the struct's placement)
-    double pp[2][TD_PLEN];     // p, permuted
+    double up[2][G * TD_PSTRIDE];   // u, permuted (16-byte aligned by the struct's placement)
+    double pp[2][G * TD_PSTRIDE];   // p, permuted
     double wsum[2][8];
-    double sspart[2][16];      // partial sums of squares of the published row, one per holder thread
-    double dg[D], of[D], ta[D];
+    double sspart[2][G];            // partial sums of squares of the published row, one per holder thread
+    double dg[8 * G], of[8 * G], ta[8 * G];
 };
 
-// The sixteen threads that hold row r (slot AR = r / 16 of their tiles) publish its raw tail
+// The G threads that hold row r (slot AR = r / G of their tiles) publish its raw tail
 // x = A[r][r+1..] into buffer `nxt`, together with their partial sums of squares of x[r+2..].  The
 // norm, beta and gamma of the reflector are worked out by every thread after the next barrier, in
-// the shadow of the matrix-vector product, instead of by these sixteen while the CTA waits.
-template <int AR>
-__device__ __forceinline__ void td_publish(const double (&A)[8][8], int r, int nxt, int tc, TdShared &sh) {
+// the shadow of the matrix-vector product, instead of by these holders while the CTA waits.
+template <int G, int AR>
+__device__ __forceinline__ void td_publish(const double (&A)[8][8], int r, int nxt, int tc, TdShared<G> &sh) {
     double x[8];
     double ss0 = 0.0, ss1 = 0.0;
 #pragma unroll
@@ -51,7 +59,7 @@ __device__ __forceinline__ void td_publish(const double (&A)[8][8], int r, int n
         if (b < AR) {
             x[b] = 0.0;
         } else {
-            const int j = tc + 16 * b;
+            const int j = tc + G * b;
             const double v = A[AR][b];
             if (b == AR && j == r) sh.dg[r] = v;
             x[b] = (j > r) ? v : 0.0;
@@ -68,22 +76,31 @@ __device__ __forceinline__ void td_publish(const double (&A)[8][8], int r, int n
     sh.sspart[nxt][tc] = ss0 + ss1;
 }
 
-// One step k with (k + 1) / 16 == K0: tile slots below K0 hold only finished rows and columns and
-// are skipped at compile time.
-template <int K0>
-__device__ __forceinline__ void td_step(double (&A)[8][8], int k, int tid, TdShared &sh, double *__restrict__ refl) {
-    const int lane = tid & 31, warp = tid >> 5, tr = tid >> 4, tc = tid & 15;
+// One step k with (k + 1) / G == K0: tile slots below K0 hold only finished rows and columns and
+// are skipped at compile time.  `refl_row` (8 G doubles of shared memory) receives the reflector.
+template <int G, int K0>
+__device__ __forceinline__ void td_step(double (&A)[8][8], int k, int tid, TdShared<G> &sh, double *__restrict__ refl_row) {
+    constexpr int N = 8 * G, NW = G * G / 32;
+    const int lane = tid & 31, warp = tid >> 5, tr = tid / G, tc = tid & (G - 1);
     __syncthreads();
     const int cur = k & 1;
     // reflector scalars from the published row: u = x - beta e_{k+1}, H = I - gamma u u^T
     double ss;
     {
         const double2 *sp = reinterpret_cast<const double2 *>(sh.sspart[cur]);
-        const double2 s0 = sp[0], s1 = sp[1], s2 = sp[2], s3 = sp[3], s4 = sp[4], s5 = sp[5], s6 = sp[6], s7 = sp[7];
-        ss = (((s0.x + s0.y) + (s1.x + s1.y)) + ((s2.x + s2.y) + (s3.x + s3.y))) +
-             (((s4.x + s4.y) + (s5.x + s5.y)) + ((s6.x + s6.y) + (s7.x + s7.y)));
+        double part[G / 2];
+#pragma unroll
+        for (int q = 0; q < G / 2; ++q) {
+            const double2 v = sp[q];
+            part[q] = v.x + v.y;
+        }
+#pragma unroll
+        for (int w = G / 4; w >= 1; w >>= 1)
+#pragma unroll
+            for (int q = 0; q < w; ++q) part[q] = part[2 * q] + part[2 * q + 1];
+        ss = part[0];
     }
-    const double alpha = sh.up[cur][td_pos(k + 1)];
+    const double alpha = sh.up[cur][td_pos<G>(k + 1)];
     double beta = alpha, gamma = 0.0;
     if (ss > 0.0) {
         const double sq = fma(alpha, alpha, ss);
@@ -91,13 +108,13 @@ __device__ __forceinline__ void td_step(double (&A)[8][8], int k, int tid, TdSha
         beta = (alpha >= 0.0) ? -nrm : nrm;
         gamma = 1.0 / fma(fabs(alpha), nrm, sq);   // 1 / (beta (beta - alpha))
     }
-    if (tid < D) refl[k * D + tid] = (tid > k) ? sh.up[cur][td_pos(tid)] - ((tid == k + 1) ? beta : 0.0) : 0.0;
+    if (tid < N) refl_row[tid] = (tid > k) ? sh.up[cur][td_pos<G>(tid)] - ((tid == k + 1) ? beta : 0.0) : 0.0;
     if (tid == 0) {
         sh.of[k] = beta;
         sh.ta[k] = gamma;
     }
-    const bool owner = (tr == ((k + 1) & 15)) && (k + 1 < D - 2);
-    const bool col_holder = tc == ((k + 1) & 15), row_holder = tr == ((k + 1) & 15);   // of index k + 1 (tile slot K0)
+    const bool owner = (tr == ((k + 1) & (G - 1))) && (k + 1 < N - 2);
+    const bool col_holder = tc == ((k + 1) & (G - 1)), row_holder = tr == ((k + 1) & (G - 1));   // of index k + 1 (tile slot K0)
     if (gamma != 0.0) {   // uniform over the CTA
         double uj[8], ui[8], acc[8];
         {
@@ -135,33 +152,40 @@ __device__ __forceinline__ void td_step(double (&A)[8][8], int k, int tid, TdSha
             if (col_holder) acc[a] = fma(-beta, A[a][K0], acc[a]);
             tloc = fma(ui[a], acc[a], tloc);
         }
-        // sum the partial rows over the sixteen column groups: each stage keeps half of the rows
-        const bool h8 = tc & 8, h4 = tc & 4, h2 = tc & 2;
+        // sum the partial rows over the G column groups: each stage keeps half of the rows
+        const bool hA = tc & (G / 2), hB = tc & (G / 4), hC = tc & (G / 8);
         double v4[4], v2[2], v1;
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-            const double keep = h8 ? acc[q + 4] : acc[q], send = h8 ? acc[q] : acc[q + 4];
-            v4[q] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+            const double keep = hA ? acc[q + 4] : acc[q], send = hA ? acc[q] : acc[q + 4];
+            v4[q] = keep + __shfl_xor_sync(0xffffffffu, send, G / 2);
         }
 #pragma unroll
         for (int q = 0; q < 2; ++q) {
-            const double keep = h4 ? v4[q + 2] : v4[q], send = h4 ? v4[q] : v4[q + 2];
-            v2[q] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+            const double keep = hB ? v4[q + 2] : v4[q], send = hB ? v4[q] : v4[q + 2];
+            v2[q] = keep + __shfl_xor_sync(0xffffffffu, send, G / 4);
         }
         {
-            const double keep = h2 ? v2[1] : v2[0], send = h2 ? v2[0] : v2[1];
-            v1 = keep + __shfl_xor_sync(0xffffffffu, send, 2);
+            const double keep = hC ? v2[1] : v2[0], send = hC ? v2[0] : v2[1];
+            v1 = keep + __shfl_xor_sync(0xffffffffu, send, G / 8);
         }
-        v1 += __shfl_xor_sync(0xffffffffu, v1, 1);
-        const int arow = (h8 ? 4 : 0) + (h4 ? 2 : 0) + (h2 ? 1 : 0);
-        const int irow = tr + 16 * arow;
-        if (!(tc & 1) && irow > k) sh.pp[cur][td_pos(irow)] = gamma * v1;
+        if (G == 16) v1 += __shfl_xor_sync(0xffffffffu, v1, 1);   // two threads per row are left: both get the sum
+        const int arow = (hA ? 4 : 0) + (hB ? 2 : 0) + (hC ? 1 : 0);
+        const int irow = tr + G * arow;
+        if ((G == 8 || !(tc & 1)) && irow > k) sh.pp[cur][td_pos<G>(irow)] = gamma * v1;
         tloc = warp_sum(tloc);
         if (lane == 0) sh.wsum[cur][warp] = tloc;
         __syncthreads();
-        const double2 w0 = *reinterpret_cast<const double2 *>(&sh.wsum[cur][0]), w1 = *reinterpret_cast<const double2 *>(&sh.wsum[cur][2]);
-        const double2 w2 = *reinterpret_cast<const double2 *>(&sh.wsum[cur][4]), w3 = *reinterpret_cast<const double2 *>(&sh.wsum[cur][6]);
-        const double uAu = ((w0.x + w0.y) + (w1.x + w1.y)) + ((w2.x + w2.y) + (w3.x + w3.y));
+        double uAu;
+        {
+            const double2 *wp = reinterpret_cast<const double2 *>(&sh.wsum[cur][0]);
+            const double2 w0 = wp[0];
+            uAu = w0.x + w0.y;
+            if (NW == 8) {
+                const double2 w1 = wp[1], w2 = wp[2], w3 = wp[3];
+                uAu = (uAu + (w1.x + w1.y)) + ((w2.x + w2.y) + (w3.x + w3.y));
+            }
+        }
         const double twoK = gamma * gamma * uAu;
         double pj[8], si[8];
         {
@@ -181,7 +205,7 @@ __device__ __forceinline__ void td_step(double (&A)[8][8], int k, int tid, TdSha
         if (owner) {
 #pragma unroll
             for (int b = K0; b < 8; ++b) A[K0][b] = fma(-ui[K0], pj[b], fma(-si[K0], uj[b], A[K0][b]));
-            td_publish<K0>(A, k + 1, cur ^ 1, tc, sh);
+            td_publish<G, K0>(A, k + 1, cur ^ 1, tc, sh);
         }
 #pragma unroll
         for (int a = K0; a < 8; ++a) {
@@ -191,69 +215,99 @@ __device__ __forceinline__ void td_step(double (&A)[8][8], int k, int tid, TdSha
             }
         }
     } else if (owner) {
-        td_publish<K0>(A, k + 1, cur ^ 1, tc, sh);
+        td_publish<G, K0>(A, k + 1, cur ^ 1, tc, sh);
     }
 }
 
-__global__ void __launch_bounds__(TD_THREADS, 1) tridiag_kernel(double *__restrict__ gram, double *__restrict__ diag,
-                                                                double *__restrict__ off, double *__restrict__ tau,
-                                                                const int *__restrict__ list, const int *__restrict__ count) {
-    extern __shared__ __align__(16) double td_refl[];   // [D][D]: staging of the matrix, then the reflectors
-    __shared__ __align__(16) TdShared sh;
-    const int tid = threadIdx.x, lane = tid & 31;
-    const int tr = tid >> 4, tc = tid & 15;
+template <int G, int K0, int LO, int HI>
+__device__ __forceinline__ void td_step_if(double (&A)[8][8], int k, int tid, TdShared<G> &sh, double *__restrict__ refl_row) {
+    if constexpr (K0 >= LO && K0 <= HI) td_step<G, K0>(A, k, tid, sh, refl_row);
+}
+
+// Steps [KB, KE) of the tridiagonalisation of the order-8G matrix whose element (i, j) sits at
+// gram[(ORIGIN + i) D + ORIGIN + j].  KB and KE are multiples of G, or KE = 8 G - 2 (the last step).
+// The trailing matrix is read from, and when steps remain written back to, its own place in
+// global memory; reflector rows ORIGIN + KB .. ORIGIN + KE - 1 then overwrite rows that are no
+// longer part of it.  Only the tile slots from KB / G up are ever live, so a kernel that starts
+// late needs fewer registers and more of its CTAs fit on an SM.
+template <int G, int ORIGIN, int KB, int KE, int MINB>
+__global__ void __launch_bounds__(G * G, MINB) tridiag_range_kernel(double *__restrict__ gram, double *__restrict__ diag,
+                                                                     double *__restrict__ off, double *__restrict__ tau,
+                                                                     const int *__restrict__ list, const int *__restrict__ count) {
+    constexpr int N = 8 * G, THREADS = G * G, S0 = KB / G;
+    constexpr bool LAST = (KE == N - 2);
+    static_assert(KB % G == 0 && (LAST || KE % G == 0), "ranges start and end on tile-slot boundaries");
+    __shared__ __align__(16) double refl[(KE - KB) * N];   // the reflectors of this range
+    __shared__ __align__(16) TdShared<G> sh;
+    const int tid = threadIdx.x;
+    const int tr = tid / G, tc = tid & (G - 1);
     int blk = blockIdx.x;
     if (list) {
         if (blk >= *count) return;
         blk = list[blk];
     }
-    double *G = gram + static_cast<size_t>(blk) * D * D;
+    double *Gm = gram + static_cast<size_t>(blk) * D * D;
+    double *T = Gm + static_cast<size_t>(ORIGIN) * D + ORIGIN;
 
-    for (int e = tid; e < D * D / 2; e += TD_THREADS)
-        reinterpret_cast<double2 *>(td_refl)[e] = reinterpret_cast<const double2 *>(G)[e];
-    if (tid < TD_PLEN) {
-        sh.up[0][tid] = 0.0;
-        sh.up[1][tid] = 0.0;
-        sh.pp[0][tid] = 0.0;
-        sh.pp[1][tid] = 0.0;
-    }
-    __syncthreads();
     double A[8][8];
 #pragma unroll
-    for (int a = 0; a < 8; ++a)
+    for (int a = S0; a < 8; ++a)
 #pragma unroll
-        for (int b = 0; b < 8; ++b) A[a][b] = td_refl[(tr + 16 * a) * D + tc + 16 * b];
+        for (int b = S0; b < 8; ++b) A[a][b] = T[static_cast<size_t>(tr + G * a) * D + tc + G * b];
+    for (int e = tid; e < G * TD_PSTRIDE; e += THREADS) {
+        sh.up[0][e] = 0.0;
+        sh.up[1][e] = 0.0;
+        sh.pp[0][e] = 0.0;
+        sh.pp[1][e] = 0.0;
+    }
     __syncthreads();
 
-    if (tr == 0) td_publish<0>(A, 0, 0, tc, sh);
+    if (tr == 0) td_publish<G, S0>(A, KB, KB & 1, tc, sh);
+    constexpr int LO = (KB + 1) / G, HI = (LAST ? KE - 1 : KE) / G;
 #pragma unroll 1
-    for (int k = 0; k < D - 2; ++k) {
-        switch ((k + 1) >> 4) {
-            case 0: td_step<0>(A, k, tid, sh, td_refl); break;
-            case 1: td_step<1>(A, k, tid, sh, td_refl); break;
-            case 2: td_step<2>(A, k, tid, sh, td_refl); break;
-            case 3: td_step<3>(A, k, tid, sh, td_refl); break;
-            case 4: td_step<4>(A, k, tid, sh, td_refl); break;
-            case 5: td_step<5>(A, k, tid, sh, td_refl); break;
-            case 6: td_step<6>(A, k, tid, sh, td_refl); break;
-            default: td_step<7>(A, k, tid, sh, td_refl); break;
+    for (int k = KB; k < KE; ++k) {
+        double *row = refl + (k - KB) * N;
+        switch ((k + 1) / G) {
+            case 0: td_step_if<G, 0, LO, HI>(A, k, tid, sh, row); break;
+            case 1: td_step_if<G, 1, LO, HI>(A, k, tid, sh, row); break;
+            case 2: td_step_if<G, 2, LO, HI>(A, k, tid, sh, row); break;
+            case 3: td_step_if<G, 3, LO, HI>(A, k, tid, sh, row); break;
+            case 4: td_step_if<G, 4, LO, HI>(A, k, tid, sh, row); break;
+            case 5: td_step_if<G, 5, LO, HI>(A, k, tid, sh, row); break;
+            case 6: td_step_if<G, 6, LO, HI>(A, k, tid, sh, row); break;
+            default: td_step_if<G, 7, LO, HI>(A, k, tid, sh, row); break;
         }
     }
-    if (tid == 14 * 16 + 14) sh.dg[D - 2] = A[7][7];
-    if (tid == 14 * 16 + 15) sh.of[D - 2] = A[7][7];
-    if (tid == 15 * 16 + 15) sh.dg[D - 1] = A[7][7];
-    if (tid == 0) {
-        sh.of[D - 1] = 0.0;
-        sh.ta[D - 2] = 0.0;
-        sh.ta[D - 1] = 0.0;
+    if (LAST) {
+        if (tid == (G - 2) * G + G - 2) sh.dg[N - 2] = A[7][7];
+        if (tid == (G - 2) * G + G - 1) sh.of[N - 2] = A[7][7];
+        if (tid == (G - 1) * G + G - 1) sh.dg[N - 1] = A[7][7];
+        if (tid == 0) {
+            sh.of[N - 1] = 0.0;
+            sh.ta[N - 2] = 0.0;
+            sh.ta[N - 1] = 0.0;
+        }
     }
     __syncthreads();
-    for (int e = tid; e < (D - 2) * D / 2; e += TD_THREADS)
-        reinterpret_cast<double2 *>(G)[e] = reinterpret_cast<const double2 *>(td_refl)[e];
-    if (tid < D) {
-        diag[static_cast<size_t>(blk) * D + tid] = sh.dg[tid];
-        off[static_cast<size_t>(blk) * D + tid] = sh.of[tid];
-        tau[static_cast<size_t>(blk) * D + tid] = sh.ta[tid];
+    // reflector of step k: zero up to column ORIGIN + k, in the full-width row ORIGIN + k
+    for (int e = tid; e < (KE - KB) * (D / 2); e += THREADS) {
+        const int r = e / (D / 2), c2 = e % (D / 2);
+        const double2 v = (c2 < ORIGIN / 2) ? make_double2(0.0, 0.0) : reinterpret_cast<const double2 *>(refl + r * N)[c2 - ORIGIN / 2];
+        reinterpret_cast<double2 *>(Gm + static_cast<size_t>(ORIGIN + KB + r) * D)[c2] = v;
+    }
+    if (!LAST) {
+        constexpr int S1 = KE / G;
+#pragma unroll
+        for (int a = S1; a < 8; ++a)
+#pragma unroll
+            for (int b = S1; b < 8; ++b) T[static_cast<size_t>(tr + G * a) * D + tc + G * b] = A[a][b];
+    }
+    constexpr int KOUT = LAST ? N : KE;
+    for (int k = KB + tid; k < KOUT; k += THREADS) {
+        const size_t o = static_cast<size_t>(blk) * D + ORIGIN + k;
+        diag[o] = sh.dg[k];
+        off[o] = sh.of[k];
+        tau[o] = sh.ta[k];
     }
 }
 
@@ -665,14 +719,16 @@ void launch_mark_redo(int64_t nb, const Workspace &ws, cudaStream_t s) {
     mark_redo_kernel<<<static_cast<unsigned>((nb + 255) / 256), 256, 0, s>>>(ws.lam, static_cast<int>(nb), ws.redo_list, ws.redo_count);
 }
 
-void launch_tridiag(int64_t nb, const Workspace &ws, const int *list, const int *count, cudaStream_t s) {
-    static bool configured = false;
-    const size_t smem = sizeof(double) * D * D;
-    if (!configured) {
-        cudaFuncSetAttribute(tridiag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-        configured = true;
+// The three ranges: order 128 with one CTA per SM while every tile slot is live, two CTAs per SM
+// from step 32, and the trailing 64 x 64 matrix on 64 threads with four CTAs per SM.
+void launch_tridiag(int part, int64_t nb, const Workspace &ws, const int *list, const int *count, cudaStream_t s) {
+    const unsigned g = static_cast<unsigned>(nb);
+    double *g0 = ws.gram, *d0 = ws.diag, *o0 = ws.off, *t0 = ws.tau;
+    switch (part) {
+        case 0: tridiag_range_kernel<16, 0, 0, 32, 1><<<g, 256, 0, s>>>(g0, d0, o0, t0, list, count); break;
+        case 1: tridiag_range_kernel<16, 0, 32, 64, 2><<<g, 256, 0, s>>>(g0, d0, o0, t0, list, count); break;
+        default: tridiag_range_kernel<8, 64, 0, 62, 4><<<g, 64, 0, s>>>(g0, d0, o0, t0, list, count); break;
     }
-    tridiag_kernel<<<static_cast<unsigned>(nb), TD_THREADS, smem, s>>>(ws.gram, ws.diag, ws.off, ws.tau, list, count);
 }
 
 void launch_eigvals(int64_t nb, const Workspace &ws, const int *list, const int *count, cudaStream_t s) {
