@@ -312,58 +312,86 @@ __global__ void __launch_bounds__(G * G, MINB) tridiag_range_kernel(double *__re
 }
 
 // ------------------------------------------------------------------------------------------
-// Eigenvalues of a symmetric tridiagonal matrix from Sturm counts: with
+// Eigenvalues of a symmetric tridiagonal matrix from Sturm sequences: with
 //   p_0 = 1, p_1 = d_0 - x, p_{i+1} = (d_i - x) p_i - e_{i-1}^2 p_{i-1},
-// the number of sign changes in p_0 .. p_d is the number of eigenvalues below x.  One thread per
-// eigenvalue.  A first pass counts at 128 points spaced geometrically below the Gershgorin bound
-// (the spectrum of a Gram matrix spans many decades), which brackets every eigenvalue to 18 %;
-// bisection then runs until the bracket is below 1e-8 relative (2e-15 of the matrix scale for the
-// smallest ones).
+// the number of sign changes in p_0 .. p_d is the number of eigenvalues below x, and p_d(x) is the
+// characteristic polynomial.  One thread per eigenvalue.  A first pass evaluates at 128 points
+// spaced geometrically below the Gershgorin bound (the spectrum of a Gram matrix spans many
+// decades), which brackets every eigenvalue to 18 %.  Each thread then shrinks its bracket until
+// it is below 1e-8 relative (2e-15 of the matrix scale for the smallest ones): by bisection on
+// the counts while the bracket holds several eigenvalues, and once it holds exactly one, by
+// regula falsi on p_d (Illinois variant: an end that survives twice has its value halved), which
+// needs a third of the evaluations.  The count still decides which end every new point replaces,
+// so a bracket never loses its eigenvalue; a step that would fall outside it is bisected instead.
 // ------------------------------------------------------------------------------------------
 constexpr double EV_E2_FLOOR = 1e-60;   // keeps the recurrence alive across an exactly decoupled entry
-constexpr int EV_MAX_BISECT = 64;
+constexpr int EV_MAX_ITER = 96;
+constexpr double EV_SECANT_WIDTH = 2e-3;   // relative bracket width below which p_d is interpolated
+constexpr int EV_PE_INVALID = -(1 << 28);   // exponent marking a p_d whose magnitude was lost
 
-// (d_i, e_{i-1}^2) pairs, scaled so that every entry is at most 1 in magnitude.
-__device__ __forceinline__ int sturm_count(const double2 *__restrict__ sde, double x) {
+constexpr int EV_GROUP = 8;               // recurrence steps between two range checks
+constexpr int EV_PAD = EV_GROUP;          // entries past the end that the look-ahead may read
+
+__device__ __forceinline__ void sturm_step(const double2 de, double x, double &p0, double &p1, unsigned &cnt) {
+    const double t = de.y * p0;
+    const double p2 = fma(de.x - x, p1, -t);
+    cnt += static_cast<unsigned>(__double2hiint(p1) ^ __double2hiint(p2)) >> 31;
+    p0 = p1;
+    p1 = p2;
+}
+
+// sde[i] = (d_i, e_{i-1}^2), scaled so that every entry is at most 1 in magnitude, followed by
+// EV_PAD entries that are read but not used.  Returns the count; p_d(x) = pm 2^pe.  The entries
+// of the next group are fetched before the current group's chain of dependent multiply-adds
+// starts, and the pair is brought back to within 2^+-300 of one after every group: eight steps
+// move it by at most 2^13 upwards and, even with full cancellation in every step, 2^-424 downwards.
+__device__ __forceinline__ int sturm_eval(const double2 *__restrict__ sde, double x, double &pm, int &pe) {
     double p0 = 1.0, p1 = sde[0].x - x;
     unsigned cnt = static_cast<unsigned>(__double2hiint(p1)) >> 31;
-#pragma unroll 1
-    for (int i0 = 1; i0 < D; i0 += 4) {
+    int esum = 0;
+    constexpr int NG = (D - 1) / EV_GROUP;
+    double2 cur[EV_GROUP], nxt[EV_GROUP];
 #pragma unroll
-        for (int i = i0; i < i0 + 4; ++i) {
-            if (i < D) {
-                const double2 de = sde[i];
-                const double t = de.y * p0;
-                const double p2 = fma(de.x - x, p1, -t);
-                cnt += static_cast<unsigned>(__double2hiint(p1) ^ __double2hiint(p2)) >> 31;
-                p0 = p1;
-                p1 = p2;
-            }
-        }
-        // keep the pair within 2^+-300 of one
+    for (int i = 0; i < EV_GROUP; ++i) cur[i] = sde[1 + i];
+#pragma unroll 1
+    for (int g = 0; g < NG; ++g) {
+        const double2 *q = sde + 1 + (g + 1) * EV_GROUP;
+#pragma unroll
+        for (int i = 0; i < EV_GROUP; ++i) nxt[i] = q[i];
+#pragma unroll
+        for (int i = 0; i < EV_GROUP; ++i) sturm_step(cur[i], x, p0, p1, cnt);
         const int e0 = (__double2hiint(p0) >> 20) & 0x7ff, e1 = (__double2hiint(p1) >> 20) & 0x7ff;
         const int em = max(e0, e1);
         if (static_cast<unsigned>(em - 723) > 600u) {
             if (em == 0) {   // both vanished: restart with the current sign
                 p0 = 0.0;
                 p1 = (__double2hiint(p1) < 0) ? -1.0 : 1.0;
+                esum = EV_PE_INVALID;
             } else if (em < 2047) {
-                const double sc = __hiloint2double((2046 - em) << 20, 0);
+                const double sc = __hiloint2double((2046 - em) << 20, 0);   // 2^(1023 - em)
                 p0 *= sc;
                 p1 *= sc;
+                esum += em - 1023;
             }
         }
+#pragma unroll
+        for (int i = 0; i < EV_GROUP; ++i) cur[i] = nxt[i];
     }
+#pragma unroll
+    for (int i = 0; i < (D - 1) - NG * EV_GROUP; ++i) sturm_step(cur[i], x, p0, p1, cnt);
+    pm = p1;
+    pe = esum;
     return static_cast<int>(cnt);
 }
 
 __global__ void __launch_bounds__(D) eigvals_kernel(const double *__restrict__ diag, const double *__restrict__ off,
                                                     double *__restrict__ lam, const int *__restrict__ list,
                                                     const int *__restrict__ count) {
-    __shared__ __align__(16) double2 sde[D];
+    __shared__ __align__(16) double2 sde[D + EV_PAD];
     __shared__ double s_e2[D];
     __shared__ double s_red[3][4];
-    __shared__ int s_cnt[D];
+    __shared__ int s_cnt[D], s_pe[D];
+    __shared__ double s_pm[D];
     const int tid = threadIdx.x;
     int blk = blockIdx.x;
     if (list) {
@@ -394,6 +422,7 @@ __global__ void __launch_bounds__(D) eigvals_kernel(const double *__restrict__ d
     __syncthreads();
     const double se_prev = (tid > 0) ? fabs(off[base + tid - 1] * scale) : 0.0;
     sde[tid] = make_double2(sd, (tid > 0) ? s_e2[tid - 1] : 0.0);
+    if (tid < EV_PAD) sde[D + tid] = make_double2(0.0, 0.0);
     // Gershgorin bounds of the scaled matrix
     double glo = sd - se - se_prev, ghi = sd + se + se_prev;
 #pragma unroll
@@ -418,7 +447,13 @@ __global__ void __launch_bounds__(D) eigvals_kernel(const double *__restrict__ d
         if (geometric) return ghi * exp2(-(9.0 * 3.321928094887362 / (D - 1)) * static_cast<double>(D - 1 - t));
         return glo + (ghi - glo) * static_cast<double>(t + 1) / static_cast<double>(D);
     };
-    s_cnt[tid] = sturm_count(sde, point(tid));
+    {
+        double pm;
+        int pe;
+        s_cnt[tid] = sturm_eval(sde, point(tid), pm, pe);
+        s_pm[tid] = pm;
+        s_pe[tid] = pe;
+    }
     __syncthreads();
     const int target = D - 1 - tid;  // ascending index of the eigenvalue this thread brackets
     int t = -1;                      // largest grid index with count <= target
@@ -427,12 +462,47 @@ __global__ void __launch_bounds__(D) eigvals_kernel(const double *__restrict__ d
         if (t + step < D && s_cnt[t + step] <= target) t += step;
     double lo = point(t), hi = (t + 1 < D) ? point(t + 1) : ghi;
     if (t == D - 1) lo = hi;   // cannot happen (every eigenvalue is below the last point); keeps the bracket sane
-    for (int it = 0; it < EV_MAX_BISECT; ++it) {
+    // counts and p_d at both ends (ends that are not grid points carry no value)
+    int clo = (t >= 0) ? s_cnt[t] : 0, chi = (t + 1 < D) ? s_cnt[t + 1] : D;
+    double flo = (t >= 0) ? s_pm[t] : 0.0, fhi = (t + 1 < D) ? s_pm[t + 1] : 0.0;
+    int elo = (t >= 0) ? s_pe[t] : EV_PE_INVALID, ehi = (t + 1 < D) ? s_pe[t + 1] : EV_PE_INVALID;
+    int replaced = 0;   // +1: the last point became hi, -1: it became lo
+    int poor = 0;
+    for (int it = 0; it < EV_MAX_ITER; ++it) {
         const double mid = 0.5 * (lo + hi);
         const bool done = (hi - lo) <= fmax(2e-15, 1e-8 * fabs(mid));
         if (__all_sync(0xffffffffu, done)) break;
-        if (sturm_count(sde, mid) > target) hi = mid;
-        else lo = mid;
+        double x = mid;
+        // p_d varies like x^d over a wide bracket, far from linear: interpolate only in a narrow one
+        if (chi - clo == 1 && poor < 3 && (hi - lo) <= EV_SECANT_WIDTH * fabs(mid) && elo > EV_PE_INVALID / 2 &&
+            ehi > EV_PE_INVALID / 2 && flo != 0.0) {
+            const double r = scalbn(fhi / flo, max(-2000, min(2000, ehi - elo)));   // p_d(hi) / p_d(lo), negative
+            if (r < 0.0) {
+                const double xs = lo + (hi - lo) / (1.0 - r);
+                if (xs > lo && xs < hi) x = xs;
+            }
+        }
+        const bool secant = x != mid;
+        const double width = hi - lo;
+        double pm;
+        int pe;
+        const int c = sturm_eval(sde, x, pm, pe);
+        if (c > target) {
+            hi = x;
+            chi = c;
+            fhi = pm;
+            ehi = pe;
+            if (secant && replaced > 0) flo *= 0.5;
+            replaced = 1;
+        } else {
+            lo = x;
+            clo = c;
+            flo = pm;
+            elo = pe;
+            if (secant && replaced < 0) fhi *= 0.5;
+            replaced = -1;
+        }
+        poor = (hi - lo > 0.5 * width) ? poor + 1 : 0;   // three steps in a row that fail to halve the bracket force a bisection
     }
     lam[base + tid] = 0.5 * (lo + hi) * m;
 }
