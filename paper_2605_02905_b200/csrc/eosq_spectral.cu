@@ -511,19 +511,38 @@ __global__ void __launch_bounds__(D) eigvals_kernel(const double *__restrict__ d
 // Algorithm 2 on the spectrum, then the kept eigenvectors by inverse iteration on the
 // tridiagonal matrix and back-transformation through the stored reflectors.
 // ------------------------------------------------------------------------------------------
-constexpr int LU_LANES = 16;
-constexpr size_t SPECTRAL_DYN_SMEM = sizeof(double) * (4 * D * LU_LANES + LU_LANES * D);
+//
+// Every phase here is a chain of dependent latencies (a pivot after a pivot, a reflector after a
+// reflector) that leaves most of the CTA idle, so the kernel is laid out for four CTAs of four warps
+// per SM, whose chains overlap: 12 columns of LU storage (the rank never exceeds the pilot k = 11)
+// and registers for three vectors per warp.
+constexpr int SP_THREADS = 128, SP_WARPS = SP_THREADS / 32;
+constexpr int LU_LANES = 12;
+static_assert(KPILOT < LU_LANES && KPILOT <= 3 * SP_WARPS, "one LU column and one warp slot per kept vector");
+constexpr size_t SPECTRAL_DYN_SMEM = sizeof(double) * 4 * D * LU_LANES;
 
-__global__ void __launch_bounds__(256) spectral_kernel(int n, Workspace ws, eosq_cache_t out, long long block0) {
+// 1 / x to about 2^-80 relative: the hardware's 20-bit estimate and two Newton steps.  Shorter than
+// the full division, which sits on the critical path of the factorisation; x is a clamped pivot,
+// far from the subnormal range the estimate flushes.
+__device__ __forceinline__ double sp_rcp(double x) {
+    double r;
+    asm("rcp.approx.ftz.f64 %0, %1;" : "=d"(r) : "d"(x));
+    double e = fma(-x, r, 1.0);
+    r = fma(r, e, r);
+    e = fma(-x, r, 1.0);
+    return fma(r, e, r);
+}
+
+__global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspace ws, eosq_cache_t out, long long block0) {
     __shared__ double lam[D], dd[D], ee[D], tt[D], atoms[D];
+    __shared__ double inv_e[D];              // reciprocals of the (clamped) subdiagonal entries
     __shared__ double s_phi[RMAX], s_sig[RMAX];
     __shared__ unsigned s_flags;
     extern __shared__ double dyn[];
-    double *lu_l = dyn;                      // multipliers            [D][16]
-    double *lu_d = dyn + D * LU_LANES;       // reciprocal pivots      [D][16]
-    double *lu_u = dyn + 2 * D * LU_LANES;   // first superdiagonal    [D][16]
-    double *lu_u2 = dyn + 3 * D * LU_LANES;  // second superdiagonal   [D][16]
-    double *yv = dyn + 4 * D * LU_LANES;     // iteration vectors      [D][16]
+    double *lu_l = dyn;                      // multipliers                      [D][12]
+    double *lu_d = dyn + D * LU_LANES;       // reciprocal pivots                [D][12]
+    double *lu_u = dyn + 2 * D * LU_LANES;   // first superdiagonal of U         [D][12]
+    double *yv = dyn + 3 * D * LU_LANES;     // iteration vectors                [D][12]
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = blockIdx.x;
@@ -569,9 +588,15 @@ __global__ void __launch_bounds__(256) spectral_kernel(int n, Workspace ws, eosq
             }
             atoms[tid] = a;
         }
+        const double floor_piv = 1.2e-16 * fmax(fabs(lam[0]), 1e-300);
+        if (tid < D) {   // pivots taken from the subdiagonal do not depend on the vector: their reciprocals are shared
+            double l = ee[tid];
+            if (!(fabs(l) >= floor_piv)) l = (l < 0.0) ? -floor_piv : floor_piv;
+            inv_e[tid] = sp_rcp(l);
+        }
         __syncthreads();
         // Step 3: Stieltjes transforms of F_e at z = lambda_i, D-transform, Eq. 9, Eq. 6.
-        for (int i = warp; i < rank; i += 8) {
+        for (int i = warp; i < rank; i += SP_WARPS) {
             const double z = lam[i];
             double ms = 0.0, msp = 0.0;
             for (int j = rank + lane; j < D; j += 32) {
@@ -616,28 +641,27 @@ __global__ void __launch_bounds__(256) spectral_kernel(int n, Workspace ws, eosq
         if (warp == 0 && lane < rank) {
             const int c = lane;
             const double mu = lam[c];
-            const double floor_piv = 1.2e-16 * fmax(fabs(lam[0]), 1e-300);
             unsigned piv[4] = {0u, 0u, 0u, 0u};
             double d_i = dd[0] - mu, u_i = ee[0];
             for (int i = 0; i < D - 1; ++i) {
                 const double l = ee[i];
                 const double d_next = dd[i + 1] - mu;
                 const double u_next = (i + 1 < D - 1) ? ee[i + 1] : 0.0;
+                // the reciprocal of the diagonal candidate starts before the pivot choice is known
+                const double ds = (fabs(d_i) >= floor_piv) ? d_i : ((d_i < 0.0) ? -floor_piv : floor_piv);
+                const double inv_d = sp_rcp(ds);
                 const bool keep = fabs(d_i) >= fabs(l);
-                double pv = keep ? d_i : l;   // the pivot; its reciprocal serves the elimination and the back substitution
-                if (!(fabs(pv) >= floor_piv)) pv = (pv < 0.0) ? -floor_piv : floor_piv;
-                const double inv = 1.0 / pv;
-                double fact, nd, nu;
+                double inv, fact, nd, nu;
                 if (keep) {
+                    inv = inv_d;   // the pivot's reciprocal serves the elimination and the back substitution
                     fact = l * inv;
                     lu_u[i * LU_LANES + c] = u_i;
-                    lu_u2[i * LU_LANES + c] = 0.0;
                     nd = d_next - fact * u_i;
                     nu = u_next;
-                } else {
+                } else {   // rows i and i + 1 change places: U gets a second superdiagonal entry, e_{i+1}
+                    inv = inv_e[i];
                     fact = d_i * inv;
                     lu_u[i * LU_LANES + c] = d_next;
-                    lu_u2[i * LU_LANES + c] = u_next;
                     nd = u_i - fact * d_next;
                     nu = -fact * u_next;
                     piv[i >> 5] |= 1u << (i & 31);
@@ -650,36 +674,83 @@ __global__ void __launch_bounds__(256) spectral_kernel(int n, Workspace ws, eosq
             if (!(fabs(d_i) >= floor_piv)) d_i = (d_i < 0.0) ? -floor_piv : floor_piv;
             lu_d[(D - 1) * LU_LANES + c] = 1.0 / d_i;
             lu_u[(D - 1) * LU_LANES + c] = 0.0;
-            lu_u2[(D - 1) * LU_LANES + c] = 0.0;
             for (int i = 0; i < D; ++i) {
                 const double f = (i + 1) * 0.6180339887498949;
                 yv[i * LU_LANES + c] = 0.5 + (f - floor(f));
             }
             double ss = 0.0;
             for (int it = 0; it < 2; ++it) {
+                // forward: apply the row interchanges and L^-1.  Entries are fetched a group of four
+                // ahead (the stores of a group never reach the entries already fetched).
                 double carry = yv[c];
-                for (int i = 0; i < D - 1; ++i) {  // forward: apply the row interchanges and L^-1
-                    const double next = yv[(i + 1) * LU_LANES + c];
-                    const double l = lu_l[i * LU_LANES + c];
-                    if ((piv[i >> 5] >> (i & 31)) & 1u) {
-                        yv[i * LU_LANES + c] = next;
-                        carry = carry - l * next;
-                    } else {
-                        yv[i * LU_LANES + c] = carry;
-                        carry = next - l * carry;
+                double ny[4], nl[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    ny[j] = yv[(1 + j) * LU_LANES + c];
+                    nl[j] = lu_l[j * LU_LANES + c];
+                }
+#pragma unroll 1
+                for (int i0 = 0; i0 < D - 1; i0 += 4) {
+                    double cy[4], cl[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        cy[j] = ny[j];
+                        cl[j] = nl[j];
+                        const int i = min(i0 + 4 + j, D - 2);
+                        ny[j] = yv[(i + 1) * LU_LANES + c];
+                        nl[j] = lu_l[i * LU_LANES + c];
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int i = i0 + j;
+                        if (i < D - 1) {
+                            if ((piv[i >> 5] >> (i & 31)) & 1u) {
+                                yv[i * LU_LANES + c] = cy[j];
+                                carry = carry - cl[j] * cy[j];
+                            } else {
+                                yv[i * LU_LANES + c] = carry;
+                                carry = cy[j] - cl[j] * carry;
+                            }
+                        }
                     }
                 }
-                double x1 = carry * lu_d[(D - 1) * LU_LANES + c];  // backward: U^-1
+                // backward: U^-1, as x_i = a_i - b_i x_{i+1} - c_i x_{i+2} with the coefficients
+                // prepared off the chain, so that one multiply-add separates consecutive entries
+                double x1 = carry * lu_d[(D - 1) * LU_LANES + c];
                 yv[(D - 1) * LU_LANES + c] = x1;
                 double x2 = 0.0;
                 ss = x1 * x1;
-                for (int i = D - 2; i >= 0; --i) {
-                    const double x = (yv[i * LU_LANES + c] - lu_u[i * LU_LANES + c] * x1 - lu_u2[i * LU_LANES + c] * x2) *
-                                     lu_d[i * LU_LANES + c];
-                    yv[i * LU_LANES + c] = x;
-                    ss += x * x;
-                    x2 = x1;
-                    x1 = x;
+                double na[4], nb[4], nc[4];
+                auto fetch = [&](int i, double &a, double &bq, double &cq) {
+                    const double dinv = lu_d[i * LU_LANES + c];
+                    const double e2 = (((piv[i >> 5] >> (i & 31)) & 1u) && i + 1 < D - 1) ? ee[i + 1] : 0.0;
+                    a = yv[i * LU_LANES + c] * dinv;
+                    bq = lu_u[i * LU_LANES + c] * dinv;
+                    cq = e2 * dinv;
+                };
+#pragma unroll
+                for (int j = 0; j < 4; ++j) fetch(D - 2 - j, na[j], nb[j], nc[j]);
+#pragma unroll 1
+                for (int i0 = D - 2; i0 >= 0; i0 -= 4) {
+                    double ca[4], cb[4], cc[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        ca[j] = na[j];
+                        cb[j] = nb[j];
+                        cc[j] = nc[j];
+                        fetch(max(i0 - 4 - j, 0), na[j], nb[j], nc[j]);
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int i = i0 - j;
+                        if (i >= 0) {
+                            const double x = fma(-cb[j], x1, fma(-cc[j], x2, ca[j]));
+                            yv[i * LU_LANES + c] = x;
+                            ss = fma(x, x, ss);
+                            x2 = x1;
+                            x1 = x;
+                        }
+                    }
                 }
             }
             if (!(ss > 0.0 && ss < 1e300)) atomicOr(&s_flags, EOSQ_BLOCK_NOT_CONVERGED);
@@ -687,70 +758,87 @@ __global__ void __launch_bounds__(256) spectral_kernel(int n, Workspace ws, eosq
     }
     __syncthreads();
 
-    // Back-transformation x = H_0 H_1 ... H_{D-3} y, one warp per pair of vectors (i, i + 8).
+    // Back-transformation x = H_0 H_1 ... H_{D-3} y; warp w takes the vectors w, w + 4, w + 8.
+    // Reflectors are applied two at a time, H_{k-1} H_k y = y - g_k u_k - g_{k-1} u_{k-1} with
+    //   g_k = t_k (u_k . y),   g_{k-1} = t_{k-1} ((u_{k-1} . y) - g_k (u_{k-1} . u_k)),
+    // so that one round of warp reductions serves two steps, and their rows are fetched from global
+    // memory two pairs ahead of use.
     const double *R = ws.gram + static_cast<size_t>(b) * D * D;
     float *vr = ws.vr + static_cast<size_t>(b) * RMAX * D;
     if (warp < rank) {
-        const int i0 = warp, i1 = warp + 8;
-        const bool two = i1 < rank;
-        double y0[4], y1[4];
+        constexpr int NV = 3;
+        double y[NV][4];
 #pragma unroll
-        for (int m = 0; m < 4; ++m) {
-            y0[m] = yv[(lane + 32 * m) * LU_LANES + i0];
-            y1[m] = two ? yv[(lane + 32 * m) * LU_LANES + i1] : 0.0;
+        for (int v = 0; v < NV; ++v) {
+            const int vi = warp + SP_WARPS * v;
+#pragma unroll
+            for (int m = 0; m < 4; ++m) y[v][m] = (vi < rank) ? yv[(lane + 32 * m) * LU_LANES + vi] : 0.0;
         }
-        // the reflector of the next step is fetched while the current one is applied
-        double nx[4];
-#pragma unroll
-        for (int m = 0; m < 4; ++m) nx[m] = R[static_cast<size_t>(D - 3) * D + lane + 32 * m];
-        for (int k = D - 3; k >= 0; --k) {
-            const double t = tt[k];
-            double vv[4], dot0 = 0.0, dot1 = 0.0;
+        double ring[2][2][4];
+        auto load_pair = [&](int k, double (&dst)[2][4]) {
 #pragma unroll
             for (int m = 0; m < 4; ++m) {
-                vv[m] = nx[m];
-                dot0 += vv[m] * y0[m];
-                dot1 += vv[m] * y1[m];
+                dst[0][m] = __ldg(R + static_cast<size_t>(k) * D + lane + 32 * m);
+                dst[1][m] = __ldg(R + static_cast<size_t>(k - 1) * D + lane + 32 * m);
             }
-            if (k > 0) {
+        };
+        load_pair(D - 3, ring[0]);
+        load_pair(D - 5, ring[1]);
+#pragma unroll 1
+        for (int k0 = D - 3; k0 >= 1; k0 -= 4) {
 #pragma unroll
-                for (int m = 0; m < 4; ++m) nx[m] = R[static_cast<size_t>(k - 1) * D + lane + 32 * m];
-            }
-            if (t == 0.0) continue;
-            dot0 = t * warp_sum(dot0);
-            dot1 = t * warp_sum(dot1);
+            for (int s2 = 0; s2 < 2; ++s2) {
+                const int k = k0 - 2 * s2;
+                if (k >= 1) {
+                    double ua[4], ub[4];
 #pragma unroll
-            for (int m = 0; m < 4; ++m) {
-                y0[m] -= dot0 * vv[m];
-                y1[m] -= dot1 * vv[m];
+                    for (int m = 0; m < 4; ++m) {
+                        ua[m] = ring[s2][0][m];
+                        ub[m] = ring[s2][1][m];
+                    }
+                    if (k - 4 >= 1) load_pair(k - 4, ring[s2]);
+                    const double ta = tt[k], tb = tt[k - 1];
+                    double dots[2 * NV + 1];
+#pragma unroll
+                    for (int v = 0; v < NV; ++v) {
+                        dots[2 * v] = fma(ua[0], y[v][0], ua[1] * y[v][1]) + fma(ua[2], y[v][2], ua[3] * y[v][3]);
+                        dots[2 * v + 1] = fma(ub[0], y[v][0], ub[1] * y[v][1]) + fma(ub[2], y[v][2], ub[3] * y[v][3]);
+                    }
+                    dots[2 * NV] = fma(ua[0], ub[0], ua[1] * ub[1]) + fma(ua[2], ub[2], ua[3] * ub[3]);
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+                        for (int q = 0; q < 2 * NV + 1; ++q) dots[q] += __shfl_xor_sync(0xffffffffu, dots[q], o);
+#pragma unroll
+                    for (int v = 0; v < NV; ++v) {
+                        const double ga = ta * dots[2 * v];
+                        const double gbb = tb * fma(-ga, dots[2 * NV], dots[2 * v + 1]);
+#pragma unroll
+                        for (int m = 0; m < 4; ++m) y[v][m] = fma(-gbb, ub[m], fma(-ga, ua[m], y[v][m]));
+                    }
+                }
             }
         }
-        double n0 = 0.0, n1 = 0.0;
 #pragma unroll
-        for (int m = 0; m < 4; ++m) {
-            n0 += y0[m] * y0[m];
-            n1 += y1[m] * y1[m];
-        }
-        n0 = warp_sum(n0);
-        n1 = warp_sum(n1);
-        const double r0 = (n0 > 0.0) ? rsqrt(n0) : 0.0, r1 = (n1 > 0.0) ? rsqrt(n1) : 0.0;
+        for (int v = 0; v < NV; ++v) {
+            const int vi = warp + SP_WARPS * v;
+            double nn = fma(y[v][0], y[v][0], y[v][1] * y[v][1]) + fma(y[v][2], y[v][2], y[v][3] * y[v][3]);
+            nn = warp_sum(nn);
+            const double rn = (nn > 0.0) ? rsqrt(nn) : 0.0;
+            if (vi < rank) {
 #pragma unroll
-        for (int m = 0; m < 4; ++m) {
-            const int j = lane + 32 * m;
-            const float f0 = static_cast<float>(y0[m] * r0);
-            vr[i0 * D + j] = f0;
-            out.V[(gb * RMAX + i0) * D + j] = __half_as_ushort(__float2half_rn(f0));
-            if (out.vr32) out.vr32[(gb * RMAX + i0) * D + j] = f0;
-            if (two) {
-                const float f1 = static_cast<float>(y1[m] * r1);
-                vr[i1 * D + j] = f1;
-                out.V[(gb * RMAX + i1) * D + j] = __half_as_ushort(__float2half_rn(f1));
-                if (out.vr32) out.vr32[(gb * RMAX + i1) * D + j] = f1;
+                for (int m = 0; m < 4; ++m) {
+                    const int j = lane + 32 * m;
+                    const float f = static_cast<float>(y[v][m] * rn);
+                    vr[vi * D + j] = f;
+                    out.V[(gb * RMAX + vi) * D + j] = __half_as_ushort(__float2half_rn(f));
+                    if (out.vr32) out.vr32[(gb * RMAX + vi) * D + j] = f;
+                }
             }
         }
     }
     // rows >= rank of V are zero; scalars
-    for (int e = tid; e < RMAX * D; e += 256) {
+    for (int e = tid; e < RMAX * D; e += SP_THREADS) {
         if (e / D >= rank) {
             out.V[gb * RMAX * D + e] = 0;
             vr[e] = 0.0f;
@@ -813,7 +901,7 @@ void launch_spectral(int64_t nb, int n, const Workspace &ws, const eosq_cache_t 
                              static_cast<int>(SPECTRAL_DYN_SMEM));
         configured = true;
     }
-    spectral_kernel<<<static_cast<unsigned>(nb), 256, SPECTRAL_DYN_SMEM, s>>>(n, ws, out, static_cast<long long>(block0));
+    spectral_kernel<<<static_cast<unsigned>(nb), SP_THREADS, SPECTRAL_DYN_SMEM, s>>>(n, ws, out, static_cast<long long>(block0));
 }
 
 }  // namespace eosq
