@@ -533,6 +533,83 @@ __device__ __forceinline__ double sp_rcp(double x) {
     return fma(r, e, r);
 }
 
+// Back-transformation of the NV vectors warp, warp + 4, .. of `yv` through the reflectors stored in
+// the rows of R, normalisation, and the stores of the kept right singular vectors.
+// Reflectors are applied two at a time, H_{k-1} H_k y = y - g_k u_k - g_{k-1} u_{k-1} with
+//   g_k = t_k (u_k . y),   g_{k-1} = t_{k-1} ((u_{k-1} . y) - g_k (u_{k-1} . u_k)),
+// so that one round of warp reductions serves two steps, and their rows are fetched from global
+// memory two pairs ahead of use.
+template <int NV>
+__device__ __forceinline__ void sp_back_transform(const double *__restrict__ R, const double *__restrict__ tt,
+                                                  const double *__restrict__ yv, int warp, int lane, float *__restrict__ vr,
+                                                  const eosq_cache_t &out, long long gb) {
+    double y[NV][4];
+#pragma unroll
+    for (int v = 0; v < NV; ++v)
+#pragma unroll
+        for (int m = 0; m < 4; ++m) y[v][m] = yv[(lane + 32 * m) * LU_LANES + warp + SP_WARPS * v];
+    double ring[2][2][4];
+    auto load_pair = [&](int k, double (&dst)[2][4]) {
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+            dst[0][m] = __ldg(R + static_cast<size_t>(k) * D + lane + 32 * m);
+            dst[1][m] = __ldg(R + static_cast<size_t>(k - 1) * D + lane + 32 * m);
+        }
+    };
+    load_pair(D - 3, ring[0]);
+    load_pair(D - 5, ring[1]);
+#pragma unroll 1
+    for (int k0 = D - 3; k0 >= 1; k0 -= 4) {
+#pragma unroll
+        for (int s2 = 0; s2 < 2; ++s2) {
+            const int k = k0 - 2 * s2;
+            if (k >= 1) {
+                double ua[4], ub[4];
+#pragma unroll
+                for (int m = 0; m < 4; ++m) {
+                    ua[m] = ring[s2][0][m];
+                    ub[m] = ring[s2][1][m];
+                }
+                if (k - 4 >= 1) load_pair(k - 4, ring[s2]);
+                const double ta = tt[k], tb = tt[k - 1];
+                double dots[2 * NV + 1];
+#pragma unroll
+                for (int v = 0; v < NV; ++v) {
+                    dots[2 * v] = fma(ua[0], y[v][0], ua[1] * y[v][1]) + fma(ua[2], y[v][2], ua[3] * y[v][3]);
+                    dots[2 * v + 1] = fma(ub[0], y[v][0], ub[1] * y[v][1]) + fma(ub[2], y[v][2], ub[3] * y[v][3]);
+                }
+                dots[2 * NV] = fma(ua[0], ub[0], ua[1] * ub[1]) + fma(ua[2], ub[2], ua[3] * ub[3]);
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+                    for (int q = 0; q < 2 * NV + 1; ++q) dots[q] += __shfl_xor_sync(0xffffffffu, dots[q], o);
+#pragma unroll
+                for (int v = 0; v < NV; ++v) {
+                    const double ga = ta * dots[2 * v];
+                    const double gbb = tb * fma(-ga, dots[2 * NV], dots[2 * v + 1]);
+#pragma unroll
+                    for (int m = 0; m < 4; ++m) y[v][m] = fma(-gbb, ub[m], fma(-ga, ua[m], y[v][m]));
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+        const int vi = warp + SP_WARPS * v;
+        double nn = fma(y[v][0], y[v][0], y[v][1] * y[v][1]) + fma(y[v][2], y[v][2], y[v][3] * y[v][3]);
+        nn = warp_sum(nn);
+        const double rn = (nn > 0.0) ? rsqrt(nn) : 0.0;
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+            const int j = lane + 32 * m;
+            const float f = static_cast<float>(y[v][m] * rn);
+            vr[vi * D + j] = f;
+            out.V[(gb * RMAX + vi) * D + j] = __half_as_ushort(__float2half_rn(f));
+            if (out.vr32) out.vr32[(gb * RMAX + vi) * D + j] = f;
+        }
+    }
+}
+
 __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspace ws, eosq_cache_t out, long long block0) {
     __shared__ double lam[D], dd[D], ee[D], tt[D], atoms[D];
     __shared__ double inv_e[D];              // reciprocals of the (clamped) subdiagonal entries
@@ -639,37 +716,51 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
         // warp 0 owns vector i (column i of the arrays).  The iterate is left unnormalised: it can
         // grow by at most 1 / floor_piv per step, and the back-transformation normalises at the end.
         if (warp == 0 && lane < rank) {
+            // A lone warp pays the full latency of every instruction, so these loops are written for
+            // few instructions per row: selects instead of branches, pointers that advance by
+            // constants, the pivot bits of 32 rows in one register.
             const int c = lane;
             const double mu = lam[c];
-            unsigned piv[4] = {0u, 0u, 0u, 0u};
+            unsigned piv[4];
             double d_i = dd[0] - mu, u_i = ee[0];
-            for (int i = 0; i < D - 1; ++i) {
-                const double l = ee[i];
-                const double d_next = dd[i + 1] - mu;
-                const double u_next = (i + 1 < D - 1) ? ee[i + 1] : 0.0;
-                // the reciprocal of the diagonal candidate starts before the pivot choice is known
-                const double ds = (fabs(d_i) >= floor_piv) ? d_i : ((d_i < 0.0) ? -floor_piv : floor_piv);
-                const double inv_d = sp_rcp(ds);
-                const bool keep = fabs(d_i) >= fabs(l);
-                double inv, fact, nd, nu;
-                if (keep) {
-                    inv = inv_d;   // the pivot's reciprocal serves the elimination and the back substitution
-                    fact = l * inv;
-                    lu_u[i * LU_LANES + c] = u_i;
-                    nd = d_next - fact * u_i;
-                    nu = u_next;
-                } else {   // rows i and i + 1 change places: U gets a second superdiagonal entry, e_{i+1}
-                    inv = inv_e[i];
-                    fact = d_i * inv;
-                    lu_u[i * LU_LANES + c] = d_next;
-                    nd = u_i - fact * d_next;
-                    nu = -fact * u_next;
-                    piv[i >> 5] |= 1u << (i & 31);
+            {
+                double *pl = lu_l + c, *pd = lu_d + c, *pu = lu_u + c;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    unsigned word = 0u;
+#pragma unroll 1
+                    for (int ii = 0; ii < 32; ii += 4) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int i = 32 * q + ii + j;
+                            if (i < D - 1) {
+                                const double l = ee[i];
+                                const double d_next = dd[i + 1] - mu;
+                                const double u_next = ee[i + 1];   // ee[D - 1] is zero
+                                // the reciprocal of the diagonal candidate starts before the pivot choice is known
+                                const double ds = (fabs(d_i) >= floor_piv) ? d_i : ((d_i < 0.0) ? -floor_piv : floor_piv);
+                                const double inv_d = sp_rcp(ds);
+                                const bool keep = fabs(d_i) >= fabs(l);
+                                // keep: row i stays.  Otherwise rows i and i + 1 change places and U gets a
+                                // second superdiagonal entry, e_{i+1}.
+                                const double inv = keep ? inv_d : inv_e[i];   // serves the elimination and the back substitution
+                                const double fact = (keep ? l : d_i) * inv;
+                                const double uu = keep ? u_i : d_next, other = keep ? d_next : u_i;
+                                pl[j * LU_LANES] = fact;
+                                pd[j * LU_LANES] = inv;
+                                pu[j * LU_LANES] = uu * inv;   // U's superdiagonal over its pivot
+                                d_i = fma(-fact, uu, other);
+                                u_i = keep ? u_next : -fact * u_next;
+                                word |= (keep ? 0u : 1u) << j;
+                            }
+                        }
+                        word = (word << 28) | (word >> 4);   // rotate: after eight groups bit r belongs to row 32 q + r
+                        pl += 4 * LU_LANES;
+                        pd += 4 * LU_LANES;
+                        pu += 4 * LU_LANES;
+                    }
+                    piv[q] = word;
                 }
-                lu_d[i * LU_LANES + c] = inv;
-                lu_l[i * LU_LANES + c] = fact;
-                d_i = nd;
-                u_i = nu;
             }
             if (!(fabs(d_i) >= floor_piv)) d_i = (d_i < 0.0) ? -floor_piv : floor_piv;
             lu_d[(D - 1) * LU_LANES + c] = 1.0 / d_i;
@@ -683,72 +774,98 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
                 // forward: apply the row interchanges and L^-1.  Entries are fetched a group of four
                 // ahead (the stores of a group never reach the entries already fetched).
                 double carry = yv[c];
-                double ny[4], nl[4];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    ny[j] = yv[(1 + j) * LU_LANES + c];
-                    nl[j] = lu_l[j * LU_LANES + c];
-                }
-#pragma unroll 1
-                for (int i0 = 0; i0 < D - 1; i0 += 4) {
-                    double cy[4], cl[4];
+                {
+                    double *py = yv + c;
+                    const double *pl = lu_l + c;
+                    double ny[4], nl[4];
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        cy[j] = ny[j];
-                        cl[j] = nl[j];
-                        const int i = min(i0 + 4 + j, D - 2);
-                        ny[j] = yv[(i + 1) * LU_LANES + c];
-                        nl[j] = lu_l[i * LU_LANES + c];
+                        ny[j] = py[(1 + j) * LU_LANES];
+                        nl[j] = pl[j * LU_LANES];
                     }
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const int i = i0 + j;
-                        if (i < D - 1) {
-                            if ((piv[i >> 5] >> (i & 31)) & 1u) {
-                                yv[i * LU_LANES + c] = cy[j];
-                                carry = carry - cl[j] * cy[j];
-                            } else {
-                                yv[i * LU_LANES + c] = carry;
-                                carry = cy[j] - cl[j] * carry;
+                    for (int q = 0; q < 4; ++q) {
+                        unsigned word = piv[q];
+#pragma unroll 1
+                        for (int ii = 0; ii < 32; ii += 4) {
+                            double cy[4], cl[4];
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                cy[j] = ny[j];
+                                cl[j] = nl[j];
+                                if (32 * q + ii + 4 + j < D - 1) {   // false only in the very last group
+                                    ny[j] = py[(5 + j) * LU_LANES];
+                                    nl[j] = pl[(4 + j) * LU_LANES];
+                                }
                             }
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                if (32 * q + ii + j < D - 1) {
+                                    const bool swap = (word >> j) & 1u;
+                                    const double a = swap ? cy[j] : carry, other = swap ? carry : cy[j];
+                                    py[j * LU_LANES] = a;
+                                    carry = fma(-cl[j], a, other);
+                                }
+                            }
+                            word >>= 4;
+                            py += 4 * LU_LANES;
+                            pl += 4 * LU_LANES;
                         }
                     }
                 }
                 // backward: U^-1, as x_i = a_i - b_i x_{i+1} - c_i x_{i+2} with the coefficients
-                // prepared off the chain, so that one multiply-add separates consecutive entries
+                // prepared off the chain, so that one multiply-add separates consecutive entries.
+                // Rows go down from D - 2 in groups of four, row 32 q + ii + 3 - j in slot j.
                 double x1 = carry * lu_d[(D - 1) * LU_LANES + c];
                 yv[(D - 1) * LU_LANES + c] = x1;
                 double x2 = 0.0;
                 ss = x1 * x1;
-                double na[4], nb[4], nc[4];
-                auto fetch = [&](int i, double &a, double &bq, double &cq) {
-                    const double dinv = lu_d[i * LU_LANES + c];
-                    const double e2 = (((piv[i >> 5] >> (i & 31)) & 1u) && i + 1 < D - 1) ? ee[i + 1] : 0.0;
-                    a = yv[i * LU_LANES + c] * dinv;
-                    bq = lu_u[i * LU_LANES + c] * dinv;
-                    cq = e2 * dinv;
-                };
+                {
+                    double *py = yv + (D - 4) * LU_LANES + c;   // row 32 q + ii of the current group
+                    const double *pd = lu_d + (D - 4) * LU_LANES + c, *pu = lu_u + (D - 4) * LU_LANES + c;
+                    const double *pe = ee + (D - 4) + 1;         // pe[r] = e_{i+1} for row i = 32 q + ii + r
+                    double ny[4], nd[4], nb[4], ne[4];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) fetch(D - 2 - j, na[j], nb[j], nc[j]);
-#pragma unroll 1
-                for (int i0 = D - 2; i0 >= 0; i0 -= 4) {
-                    double ca[4], cb[4], cc[4];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        ca[j] = na[j];
-                        cb[j] = nb[j];
-                        cc[j] = nc[j];
-                        fetch(max(i0 - 4 - j, 0), na[j], nb[j], nc[j]);
+                    for (int j = 1; j < 4; ++j) {   // slot 0 of the first group would be row D - 1
+                        ny[j] = py[(3 - j) * LU_LANES];
+                        nd[j] = pd[(3 - j) * LU_LANES];
+                        nb[j] = pu[(3 - j) * LU_LANES];
+                        ne[j] = pe[3 - j];
                     }
+                    ny[0] = nd[0] = nb[0] = ne[0] = 0.0;
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const int i = i0 - j;
-                        if (i >= 0) {
-                            const double x = fma(-cb[j], x1, fma(-cc[j], x2, ca[j]));
-                            yv[i * LU_LANES + c] = x;
-                            ss = fma(x, x, ss);
-                            x2 = x1;
-                            x1 = x;
+                    for (int q = 3; q >= 0; --q) {
+                        const unsigned word = piv[q];
+#pragma unroll 1
+                        for (int ii = 28; ii >= 0; ii -= 4) {
+                            const unsigned bits = word >> ii;
+                            double ca[4], cb[4], cc[4];
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                ca[j] = ny[j] * nd[j];
+                                cb[j] = nb[j];
+                                cc[j] = ((bits >> (3 - j)) & 1u) ? ne[j] * nd[j] : 0.0;
+                                if (32 * q + ii >= 4) {   // false only in the very last group
+                                    ny[j] = py[(-1 - j) * LU_LANES];
+                                    nd[j] = pd[(-1 - j) * LU_LANES];
+                                    nb[j] = pu[(-1 - j) * LU_LANES];
+                                    ne[j] = pe[-1 - j];
+                                }
+                            }
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                if (32 * q + ii + 3 - j <= D - 2) {
+                                    const double x = fma(-cb[j], x1, fma(-cc[j], x2, ca[j]));
+                                    py[(3 - j) * LU_LANES] = x;
+                                    ss = fma(x, x, ss);
+                                    x2 = x1;
+                                    x1 = x;
+                                }
+                            }
+                            py -= 4 * LU_LANES;
+                            pd -= 4 * LU_LANES;
+                            pu -= 4 * LU_LANES;
+                            pe -= 4;
                         }
                     }
                 }
@@ -758,84 +875,15 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
     }
     __syncthreads();
 
-    // Back-transformation x = H_0 H_1 ... H_{D-3} y; warp w takes the vectors w, w + 4, w + 8.
-    // Reflectors are applied two at a time, H_{k-1} H_k y = y - g_k u_k - g_{k-1} u_{k-1} with
-    //   g_k = t_k (u_k . y),   g_{k-1} = t_{k-1} ((u_{k-1} . y) - g_k (u_{k-1} . u_k)),
-    // so that one round of warp reductions serves two steps, and their rows are fetched from global
-    // memory two pairs ahead of use.
+    // Back-transformation x = H_0 H_1 ... H_{D-3} y; warp w takes those of the vectors w, w + 4, w + 8
+    // that exist (the instruction count follows the number of vectors, so it is a template argument).
     const double *R = ws.gram + static_cast<size_t>(b) * D * D;
     float *vr = ws.vr + static_cast<size_t>(b) * RMAX * D;
     if (warp < rank) {
-        constexpr int NV = 3;
-        double y[NV][4];
-#pragma unroll
-        for (int v = 0; v < NV; ++v) {
-            const int vi = warp + SP_WARPS * v;
-#pragma unroll
-            for (int m = 0; m < 4; ++m) y[v][m] = (vi < rank) ? yv[(lane + 32 * m) * LU_LANES + vi] : 0.0;
-        }
-        double ring[2][2][4];
-        auto load_pair = [&](int k, double (&dst)[2][4]) {
-#pragma unroll
-            for (int m = 0; m < 4; ++m) {
-                dst[0][m] = __ldg(R + static_cast<size_t>(k) * D + lane + 32 * m);
-                dst[1][m] = __ldg(R + static_cast<size_t>(k - 1) * D + lane + 32 * m);
-            }
-        };
-        load_pair(D - 3, ring[0]);
-        load_pair(D - 5, ring[1]);
-#pragma unroll 1
-        for (int k0 = D - 3; k0 >= 1; k0 -= 4) {
-#pragma unroll
-            for (int s2 = 0; s2 < 2; ++s2) {
-                const int k = k0 - 2 * s2;
-                if (k >= 1) {
-                    double ua[4], ub[4];
-#pragma unroll
-                    for (int m = 0; m < 4; ++m) {
-                        ua[m] = ring[s2][0][m];
-                        ub[m] = ring[s2][1][m];
-                    }
-                    if (k - 4 >= 1) load_pair(k - 4, ring[s2]);
-                    const double ta = tt[k], tb = tt[k - 1];
-                    double dots[2 * NV + 1];
-#pragma unroll
-                    for (int v = 0; v < NV; ++v) {
-                        dots[2 * v] = fma(ua[0], y[v][0], ua[1] * y[v][1]) + fma(ua[2], y[v][2], ua[3] * y[v][3]);
-                        dots[2 * v + 1] = fma(ub[0], y[v][0], ub[1] * y[v][1]) + fma(ub[2], y[v][2], ub[3] * y[v][3]);
-                    }
-                    dots[2 * NV] = fma(ua[0], ub[0], ua[1] * ub[1]) + fma(ua[2], ub[2], ua[3] * ub[3]);
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1)
-#pragma unroll
-                        for (int q = 0; q < 2 * NV + 1; ++q) dots[q] += __shfl_xor_sync(0xffffffffu, dots[q], o);
-#pragma unroll
-                    for (int v = 0; v < NV; ++v) {
-                        const double ga = ta * dots[2 * v];
-                        const double gbb = tb * fma(-ga, dots[2 * NV], dots[2 * v + 1]);
-#pragma unroll
-                        for (int m = 0; m < 4; ++m) y[v][m] = fma(-gbb, ub[m], fma(-ga, ua[m], y[v][m]));
-                    }
-                }
-            }
-        }
-#pragma unroll
-        for (int v = 0; v < NV; ++v) {
-            const int vi = warp + SP_WARPS * v;
-            double nn = fma(y[v][0], y[v][0], y[v][1] * y[v][1]) + fma(y[v][2], y[v][2], y[v][3] * y[v][3]);
-            nn = warp_sum(nn);
-            const double rn = (nn > 0.0) ? rsqrt(nn) : 0.0;
-            if (vi < rank) {
-#pragma unroll
-                for (int m = 0; m < 4; ++m) {
-                    const int j = lane + 32 * m;
-                    const float f = static_cast<float>(y[v][m] * rn);
-                    vr[vi * D + j] = f;
-                    out.V[(gb * RMAX + vi) * D + j] = __half_as_ushort(__float2half_rn(f));
-                    if (out.vr32) out.vr32[(gb * RMAX + vi) * D + j] = f;
-                }
-            }
-        }
+        const int nv = (rank - warp + SP_WARPS - 1) / SP_WARPS;
+        if (nv == 1) sp_back_transform<1>(R, tt, yv, warp, lane, vr, out, gb);
+        else if (nv == 2) sp_back_transform<2>(R, tt, yv, warp, lane, vr, out, gb);
+        else sp_back_transform<3>(R, tt, yv, warp, lane, vr, out, gb);
     }
     // rows >= rank of V are zero; scalars
     for (int e = tid; e < RMAX * D; e += SP_THREADS) {
