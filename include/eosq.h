@@ -205,12 +205,17 @@ int64_t eosq_launch_count(const eosq_ctx *ctx);
  * CUDA events on the launching stream.  eosq_profile_read synchronises those events, adds their
  * elapsed milliseconds into ms[EOSQ_NUM_STAGES] and their launch counts into
  * launches[EOSQ_NUM_STAGES] (host arrays, overwritten), and clears the record.
- * Stage order: Gram, tridiagonalisation (first 64 steps), tridiagonalisation (trailing 64 x 64
- * matrix), eigenvalues, spectrum + shrinkage + eigenvectors,
- * residual/rotate/quantise/pack, decode, scores.
+ * Stage order: Gram, tridiagonalisation steps 0-31, 32-63 and 64-125 (three kernels), eigenvalues,
+ * spectrum + shrinkage + eigenvectors, residual/rotate/quantise/pack, decode, scores, the second
+ * pass over blocks whose tensor-core Gram matrix was not accurate enough (all its kernels), other.
  */
-#define EOSQ_NUM_STAGES 9
+#define EOSQ_NUM_STAGES 11
 int eosq_profile_enable(eosq_ctx *ctx, int on);
+/* Times only the stages whose bit (1 << stage index, in the order above) is set in stage_mask; the
+ * two events per launch cost about 2 us of device time each, which adds up over the several hundred
+ * launches of a large encode, so a benchmark that wants one kernel's duration inside its timed
+ * region selects that stage alone.  EOSQ_ERR_INVALID_ARG for bits beyond EOSQ_NUM_STAGES. */
+int eosq_profile_select(eosq_ctx *ctx, uint32_t stage_mask);
 int eosq_profile_read(eosq_ctx *ctx, float *ms, int64_t *launches);
 
 #ifdef __cplusplus

@@ -26,10 +26,10 @@ EXPORTS = [
     "eosq_pilot_k", "eosq_codebook", "eosq_rotation", "eosq_layout", "eosq_bits_per_entry",
     "eosq_workspace_bytes", "eosq_create", "eosq_destroy", "eosq_last_cuda_error", "eosq_encode",
     "eosq_decode", "eosq_scores", "eosq_encode_host_arena_bytes", "eosq_encode_host",
-    "eosq_check_status", "eosq_launch_count", "eosq_profile_enable", "eosq_profile_read",
+    "eosq_check_status", "eosq_launch_count", "eosq_profile_enable", "eosq_profile_select", "eosq_profile_read",
     "eosq_encode_static", "eosq_encode_static_max_blocks",
 ]
-STAGES = ["gram", "tridiag_head", "tridiag_tail", "eigvals", "spectral", "quant", "decode", "scores", "other"]
+STAGES = ["gram", "tridiag_a", "tridiag_b", "tridiag_c", "eigvals", "spectral", "quant", "decode", "scores", "redo", "other"]
 
 
 class EosqError(RuntimeError):
@@ -91,6 +91,7 @@ def lib():
         L.eosq_encode_host.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
                                        ctypes.c_int, ctypes.c_uint64, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
         L.eosq_profile_enable.argtypes = [ctypes.c_void_p, ctypes.c_int]
+        L.eosq_profile_select.argtypes = [ctypes.c_void_p, ctypes.c_uint32]
         L.eosq_profile_read.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         L.eosq_check_status.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p]
         _lib = L
@@ -169,6 +170,13 @@ class Context:
 
     def profile_enable(self, on: bool = True):
         _check(lib().eosq_profile_enable(self._h, int(bool(on))), "eosq_profile_enable", self)
+
+    def profile_select(self, stages):
+        """Times only the named stages (see STAGES)."""
+        mask = 0
+        for name in stages:
+            mask |= 1 << STAGES.index(name)
+        _check(lib().eosq_profile_select(self._h, mask), "eosq_profile_select", self)
 
     def profile_read(self) -> dict:
         """{stage: (milliseconds, launches)} accumulated since the last read (synchronises)."""

@@ -93,7 +93,7 @@ cudaEvent_t take_event(eosq_ctx *ctx) {
 // on, bracketing it with events.
 template <typename F>
 void run_stage(eosq_ctx *ctx, int stage, cudaStream_t s, F &&launch) {
-    if (ctx->profile) {
+    if ((ctx->profile_mask >> stage) & 1u) {
         eosq_ctx::Timed t{stage, take_event(ctx), take_event(ctx)};
         cudaEventRecord(t.start, s);
         launch();
@@ -119,6 +119,10 @@ int eosq::encode_chunk(eosq_ctx *ctx, const void *blocks, int in_dtype, int64_t 
     const size_t esize = (in_dtype == EOSQ_F32) ? 4 : 2;
     const char *chunk_in = static_cast<const char *>(blocks) + static_cast<size_t>(b0) * n * D * esize;
     const eosq_cache_t o = shifted(out_all, b0, n, bits);
+    // The queue of blocks for the second pass must be empty when the eigenvalue kernel runs.  Every
+    // chunk leaves it empty (the spectral kernel clears it); the first chunk of a call cannot know
+    // what the scratch held before.
+    if (b0 == 0 && record_cuda(ctx, cudaMemsetAsync(ws.redo_count, 0, sizeof(int), s), "cudaMemsetAsync(redo count)")) return EOSQ_ERR_CUDA;
     if (in_dtype == EOSQ_F16) {
         bool setup_ok = true;
         run_stage(ctx, ST_GRAM, s, [&] { setup_ok = launch_gram_tc(blocks, 0, b0, nb, n, ws.gram, ctx->dev_err, ctx->sm_count, s); });
@@ -129,18 +133,17 @@ int eosq::encode_chunk(eosq_ctx *ctx, const void *blocks, int in_dtype, int64_t 
     } else {
         run_stage(ctx, ST_GRAM, s, [&] { launch_gram_plain(chunk_in, in_dtype, nb, n, ws.gram, nullptr, nullptr, s); });
     }
+    static_assert(TRIDIAG_PARTS == 3, "one profiling stage per tridiagonalisation kernel");
     for (int part = 0; part < TRIDIAG_PARTS; ++part)
-        run_stage(ctx, part + 1 < TRIDIAG_PARTS ? ST_TRIDIAG_HEAD : ST_TRIDIAG_TAIL, s, [&] { launch_tridiag(part, nb, ws, nullptr, nullptr, s); });
-    run_stage(ctx, ST_EIGVALS, s, [&] { launch_eigvals(nb, ws, nullptr, nullptr, s); });
+        run_stage(ctx, ST_TRIDIAG_A + part, s, [&] { launch_tridiag(part, nb, ws, nullptr, nullptr, s); });
+    // the eigenvalue kernel also queues, in ws.redo_list, the blocks the tensor-core Gram matrix cannot resolve
+    run_stage(ctx, ST_EIGVALS, s, [&] { launch_eigvals(nb, ws, nullptr, nullptr, (in_dtype == EOSQ_F16) ? ws.redo_list : nullptr, s); });
     if (in_dtype == EOSQ_F16) {
-        // second pass, exact Gram matrix, for the blocks the tensor-core one cannot resolve
-        if (record_cuda(ctx, cudaMemsetAsync(ws.redo_count, 0, sizeof(int), s), "cudaMemsetAsync(redo count)")) return EOSQ_ERR_CUDA;
-        run_stage(ctx, ST_OTHER, s, [&] { launch_mark_redo(nb, ws, s); });
-        run_stage(ctx, ST_GRAM, s, [&] { launch_gram_plain(chunk_in, in_dtype, nb, n, ws.gram, ws.redo_list, ws.redo_count, s); });
+        // second pass, exact Gram matrix, for those blocks (the spectral kernel clears the queue afterwards)
+        run_stage(ctx, ST_REDO, s, [&] { launch_gram_plain(chunk_in, in_dtype, nb, n, ws.gram, ws.redo_list, ws.redo_count, s); });
         for (int part = 0; part < TRIDIAG_PARTS; ++part)
-            run_stage(ctx, part + 1 < TRIDIAG_PARTS ? ST_TRIDIAG_HEAD : ST_TRIDIAG_TAIL, s,
-                      [&] { launch_tridiag(part, nb, ws, ws.redo_list, ws.redo_count, s); });
-        run_stage(ctx, ST_EIGVALS, s, [&] { launch_eigvals(nb, ws, ws.redo_list, ws.redo_count, s); });
+            run_stage(ctx, ST_REDO, s, [&] { launch_tridiag(part, nb, ws, ws.redo_list, ws.redo_count, s); });
+        run_stage(ctx, ST_REDO, s, [&] { launch_eigvals(nb, ws, ws.redo_list, ws.redo_count, nullptr, s); });
     }
     run_stage(ctx, ST_SPECTRAL, s, [&] { launch_spectral(nb, n, ws, o, 0, s); });
     if (in_dtype == EOSQ_F16) {
@@ -200,7 +203,13 @@ extern "C" int eosq_destroy(eosq_ctx *ctx) {
 
 extern "C" int eosq_profile_enable(eosq_ctx *ctx, int on) {
     if (!ctx) return EOSQ_ERR_INVALID_ARG;
-    ctx->profile = on != 0;
+    ctx->profile_mask = on ? ((1u << EOSQ_NUM_STAGES) - 1u) : 0u;
+    return EOSQ_OK;
+}
+
+extern "C" int eosq_profile_select(eosq_ctx *ctx, uint32_t stage_mask) {
+    if (!ctx || (stage_mask >> EOSQ_NUM_STAGES)) return EOSQ_ERR_INVALID_ARG;
+    ctx->profile_mask = stage_mask;
     return EOSQ_OK;
 }
 

@@ -83,7 +83,7 @@ inline size_t carve(void *base, int64_t cap, Workspace *ws) {
 
 }  // namespace eosq
 
-enum Stage { ST_GRAM = 0, ST_TRIDIAG_HEAD, ST_TRIDIAG_TAIL, ST_EIGVALS, ST_SPECTRAL, ST_QUANT, ST_DECODE, ST_SCORES, ST_OTHER };
+enum Stage { ST_GRAM = 0, ST_TRIDIAG_A, ST_TRIDIAG_B, ST_TRIDIAG_C, ST_EIGVALS, ST_SPECTRAL, ST_QUANT, ST_DECODE, ST_SCORES, ST_REDO, ST_OTHER };
 
 struct eosq_ctx {
     struct Timed {
@@ -96,7 +96,7 @@ struct eosq_ctx {
     std::vector<eosq::Rotation> rotations;
     std::string last_error;
     int64_t launches = 0;
-    bool profile = false;
+    uint32_t profile_mask = 0;   // bit i set: launches of stage i are bracketed by events
     std::vector<Timed> timed;
     std::vector<cudaEvent_t> free_events;
 };
@@ -120,12 +120,17 @@ void launch_gram_plain(const void *blocks, int in_dtype, int64_t nb, int n, doub
 bool launch_gram_tc(const void *blocks_all, int64_t nb_all, int64_t block0, int64_t nb, int n, double *gram, int *err,
                     int sm_count, cudaStream_t s);
 // Householder tridiagonalisation of each Gram matrix (in place: reflectors overwrite it).
+// Grid of a kernel that works through blocks [0, nb), or, with a list, through the few listed
+// blocks: those launches are almost always empty, and a small grid keeps them cheap.
+constexpr int64_t LIST_GRID = 148;
+inline unsigned list_grid(int64_t nb, const int *list) {
+    return static_cast<unsigned>(list ? (nb < LIST_GRID ? nb : LIST_GRID) : nb);
+}
 constexpr int TRIDIAG_PARTS = 3;
 void launch_tridiag(int part, int64_t nb, const Workspace &ws, const int *list, const int *count, cudaStream_t s);
 // All eigenvalues of each tridiagonal matrix by Sturm bisection.
-void launch_eigvals(int64_t nb, const Workspace &ws, const int *list, const int *count, cudaStream_t s);
+void launch_eigvals(int64_t nb, const Workspace &ws, const int *list, const int *count, int *mark_list, cudaStream_t s);
 // Clears the redo list / appends every block whose eigenvalue range exceeds 1 / REDO_RATIO.
-void launch_mark_redo(int64_t nb, const Workspace &ws, cudaStream_t s);
 // Bulk edge, rank, imputed spectrum, D-transform and shrinkage; kept eigenvectors.
 void launch_spectral(int64_t nb, int n, const Workspace &ws, const eosq_cache_t &out, int64_t block0,
                      cudaStream_t s);

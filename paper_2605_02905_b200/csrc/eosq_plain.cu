@@ -19,11 +19,9 @@ __global__ void __launch_bounds__(256) gram_plain_kernel(const Tin *__restrict__
                                                          const int *__restrict__ count) {
     __shared__ __align__(16) float tile[GRAM_ROWS][D];
     const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-    int blk = blockIdx.x;
-    if (list) {
-        if (blk >= *count) return;
-        blk = list[blk];
-    }
+    // without a list: block blockIdx.x; with one: the listed blocks, shared out over the grid
+    for (int li = blockIdx.x; !list || li < *count; li += gridDim.x) {
+    const int blk = list ? list[li] : li;
     const Tin *S = blocks + static_cast<size_t>(blk) * n * D;
     double acc[8][8];
 #pragma unroll
@@ -60,14 +58,16 @@ __global__ void __launch_bounds__(256) gram_plain_kernel(const Tin *__restrict__
             G[row * D + col] = acc[i][j];
         }
     }
+    if (!list) break;
+    }
 }
 
 void launch_gram_plain(const void *blocks, int in_dtype, int64_t nb, int n, double *gram, const int *list,
                        const int *count, cudaStream_t s) {
     if (in_dtype == EOSQ_F32)
-        gram_plain_kernel<float><<<static_cast<unsigned>(nb), 256, 0, s>>>(static_cast<const float *>(blocks), n, gram, list, count);
+        gram_plain_kernel<float><<<list_grid(nb, list), 256, 0, s>>>(static_cast<const float *>(blocks), n, gram, list, count);
     else
-        gram_plain_kernel<__half><<<static_cast<unsigned>(nb), 256, 0, s>>>(static_cast<const __half *>(blocks), n, gram, list, count);
+        gram_plain_kernel<__half><<<list_grid(nb, list), 256, 0, s>>>(static_cast<const __half *>(blocks), n, gram, list, count);
 }
 
 // ------------------------------------------------------------------------------------------

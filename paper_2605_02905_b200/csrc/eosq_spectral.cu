@@ -241,11 +241,9 @@ __global__ void __launch_bounds__(G * G, MINB) tridiag_range_kernel(double *__re
     __shared__ __align__(16) TdShared<G> sh;
     const int tid = threadIdx.x;
     const int tr = tid / G, tc = tid & (G - 1);
-    int blk = blockIdx.x;
-    if (list) {
-        if (blk >= *count) return;
-        blk = list[blk];
-    }
+    // without a list: block blockIdx.x; with one: the listed blocks, shared out over the grid
+    for (int li = blockIdx.x; !list || li < *count; li += gridDim.x) {
+    const int blk = list ? list[li] : li;
     double *Gm = gram + static_cast<size_t>(blk) * D * D;
     double *T = Gm + static_cast<size_t>(ORIGIN) * D + ORIGIN;
 
@@ -308,6 +306,9 @@ __global__ void __launch_bounds__(G * G, MINB) tridiag_range_kernel(double *__re
         diag[o] = sh.dg[k];
         off[o] = sh.of[k];
         tau[o] = sh.ta[k];
+    }
+    if (!list) break;
+    __syncthreads();   // the shared state is reused by the next listed block
     }
 }
 
@@ -384,20 +385,18 @@ __device__ __forceinline__ int sturm_eval(const double2 *__restrict__ sde, doubl
     return static_cast<int>(cnt);
 }
 
-__global__ void __launch_bounds__(D) eigvals_kernel(const double *__restrict__ diag, const double *__restrict__ off,
-                                                    double *__restrict__ lam, const int *__restrict__ list,
-                                                    const int *__restrict__ count) {
+// With `mark_list` set (first pass over tensor-core Gram matrices), a block whose smallest
+// eigenvalue is not at least REDO_RATIO of the largest (this includes non-finite spectra) is queued
+// in mark_list[atomicAdd(mark_count)] for a second pass with the exact Gram matrix.
+__device__ __forceinline__ void eigvals_block(const double *__restrict__ diag, const double *__restrict__ off,
+                                              double *__restrict__ lam, int blk, int *__restrict__ mark_list,
+                                              int *__restrict__ mark_count) {
     __shared__ __align__(16) double2 sde[D + EV_PAD];
     __shared__ double s_e2[D];
     __shared__ double s_red[3][4];
     __shared__ int s_cnt[D], s_pe[D];
     __shared__ double s_pm[D];
     const int tid = threadIdx.x;
-    int blk = blockIdx.x;
-    if (list) {
-        if (blk >= *count) return;
-        blk = list[blk];
-    }
     const size_t base = static_cast<size_t>(blk) * D;
     const double d0 = diag[base + tid];
     const double e0 = (tid < D - 1) ? off[base + tid] : 0.0;
@@ -409,6 +408,7 @@ __global__ void __launch_bounds__(D) eigvals_kernel(const double *__restrict__ d
     const int bad = __syncthreads_or(!(fabs(d0) < 1e300) || !(fabs(e0) < 1e300));
     if (bad) {
         lam[base + tid] = nan("");
+        if (mark_list && tid == 0) mark_list[atomicAdd(mark_count, 1)] = blk;
         return;
     }
     m = fmax(fmax(s_red[0][0], s_red[0][1]), fmax(s_red[0][2], s_red[0][3]));
@@ -504,7 +504,25 @@ __global__ void __launch_bounds__(D) eigvals_kernel(const double *__restrict__ d
         }
         poor = (hi - lo > 0.5 * width) ? poor + 1 : 0;   // three steps in a row that fail to halve the bracket force a bisection
     }
-    lam[base + tid] = 0.5 * (lo + hi) * m;
+    const double ev = 0.5 * (lo + hi) * m;
+    lam[base + tid] = ev;
+    if (mark_list) {   // uniform over the CTA
+        if (tid == 0) s_red[0][0] = ev;   // the largest eigenvalue
+        __syncthreads();
+        if (tid == D - 1 && !(ev >= REDO_RATIO * s_red[0][0])) mark_list[atomicAdd(mark_count, 1)] = blk;
+    }
+}
+
+__global__ void __launch_bounds__(D) eigvals_kernel(const double *__restrict__ diag, const double *__restrict__ off,
+                                                    double *__restrict__ lam, const int *__restrict__ list,
+                                                    const int *__restrict__ count, int *__restrict__ mark_list,
+                                                    int *__restrict__ mark_count) {
+    // without a list: block blockIdx.x; with one: the listed blocks, shared out over the grid
+    for (int li = blockIdx.x; !list || li < *count; li += gridDim.x) {
+        eigvals_block(diag, off, lam, list ? list[li] : li, mark_list, mark_count);
+        if (!list) break;
+        __syncthreads();   // the shared state is reused by the next listed block
+    }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -904,6 +922,7 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
     }
     if (tid < D && out.eig) out.eig[gb * D + tid] = static_cast<float>(lam[tid]);
     if (tid == 0) {
+        if (b == 0) *ws.redo_count = 0;   // the second pass of this chunk is over: empty its queue for the next chunk
         out.rank[gb] = rank;
         ws.rank[b] = rank;
         out.status[gb] = static_cast<int32_t>(s_flags);
@@ -911,24 +930,10 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
     }
 }
 
-// ------------------------------------------------------------------------------------------
-// Blocks whose smallest eigenvalue is not at least REDO_RATIO of the largest (this includes
-// non-finite spectra) are queued for a second pass with the exact Gram matrix.
-__global__ void mark_redo_kernel(const double *__restrict__ lam, int nb, int *__restrict__ list, int *__restrict__ count) {
-    const int b = blockIdx.x * blockDim.x + threadIdx.x;
-    if (b >= nb) return;
-    const double hi = lam[static_cast<size_t>(b) * D], lo = lam[static_cast<size_t>(b) * D + D - 1];
-    if (!(lo >= REDO_RATIO * hi)) list[atomicAdd(count, 1)] = b;
-}
-
-void launch_mark_redo(int64_t nb, const Workspace &ws, cudaStream_t s) {
-    mark_redo_kernel<<<static_cast<unsigned>((nb + 255) / 256), 256, 0, s>>>(ws.lam, static_cast<int>(nb), ws.redo_list, ws.redo_count);
-}
-
 // The three ranges: order 128 with one CTA per SM while every tile slot is live, two CTAs per SM
 // from step 32, and the trailing 64 x 64 matrix on 64 threads with four CTAs per SM.
 void launch_tridiag(int part, int64_t nb, const Workspace &ws, const int *list, const int *count, cudaStream_t s) {
-    const unsigned g = static_cast<unsigned>(nb);
+    const unsigned g = list_grid(nb, list);
     double *g0 = ws.gram, *d0 = ws.diag, *o0 = ws.off, *t0 = ws.tau;
     switch (part) {
         case 0: tridiag_range_kernel<16, 0, 0, 32, 1><<<g, 256, 0, s>>>(g0, d0, o0, t0, list, count); break;
@@ -937,8 +942,8 @@ void launch_tridiag(int part, int64_t nb, const Workspace &ws, const int *list, 
     }
 }
 
-void launch_eigvals(int64_t nb, const Workspace &ws, const int *list, const int *count, cudaStream_t s) {
-    eigvals_kernel<<<static_cast<unsigned>(nb), D, 0, s>>>(ws.diag, ws.off, ws.lam, list, count);
+void launch_eigvals(int64_t nb, const Workspace &ws, const int *list, const int *count, int *mark_list, cudaStream_t s) {
+    eigvals_kernel<<<list_grid(nb, list), D, 0, s>>>(ws.diag, ws.off, ws.lam, list, count, mark_list, ws.redo_count);
 }
 
 void launch_spectral(int64_t nb, int n, const Workspace &ws, const eosq_cache_t &out, int64_t block0,
