@@ -126,13 +126,13 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
     if (tid == 0) {
         for (int s = 0; s < WS_STAGES; ++s) {
             mbar_init(&bars.st_full[s], 1);
-            mbar_init(&bars.st_empty[s], 128 * WS_TPS);
+            mbar_init(&bars.st_empty[s], 4 * WS_TPS);   // one arrival per expander warp and tile slot
         }
         for (int b = 0; b < WS_BUFS; ++b) {
-            mbar_init(&bars.a_full[b], 128);
+            mbar_init(&bars.a_full[b], 4);             // one arrival per warp: 128 arrivals on one barrier serialise
             mbar_init(&bars.a_empty[b], 1);
             mbar_init(&bars.d_full[b], 1);
-            mbar_init(&bars.d_empty[b], 128);
+            mbar_init(&bars.d_empty[b], 4);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&bars.blk_full[b], 1);
@@ -404,7 +404,9 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
                 {   // a stage is released by 128 arrivals per tile slot; the last tile of a short stage makes up the rest
                     const int last_in_stage = min(tiles, (tile / WS_TPS + 1) * WS_TPS) - 1;
                     const int arrivals = (tile == last_in_stage) ? 1 + (WS_TPS - 1 - (tile % WS_TPS)) : 1;
-                    for (int r = 0; r < arrivals; ++r) mbar_arrive(&bars.st_empty[stage]);
+                    __syncwarp();   // every lane has its copy of the stage's bytes in registers
+                    if (lane == 0)
+                        for (int r = 0; r < arrivals; ++r) mbar_arrive(&bars.st_empty[stage]);
                 }
                 if (!valid) {   // rows past the end of the block were not copied: the stage holds stale bytes there
                     c0 = make_uint4(0u, 0u, 0u, 0u);
@@ -440,7 +442,8 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
                 }
                 tmem_st_wait();
                 tc_fence_before_sync();
-                mbar_arrive(&bars.a_full[buf]);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars.a_full[buf]);
             }
         }
     } else {
@@ -468,7 +471,8 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
                 tmem_ld8(tb + WS_COL_RHO, rv);
                 tmem_ld_wait();
                 tc_fence_before_sync();
-                mbar_arrive(&bars.d_empty[buf]);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars.d_empty[buf]);
                 const int tok = tile * 128 + wt;
                 if (tok < n) {
                     const float f1 = a.scale * __uint_as_float(rv[0]) * a.inv_code;

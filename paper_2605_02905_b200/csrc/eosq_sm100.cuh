@@ -37,16 +37,31 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
     return ok != 0;
 }
 
+// Non-blocking test of the phase: a few tens of cycles, where try_wait, which may suspend the
+// thread, costs about 200 even when the phase completed long ago.
+__device__ __forceinline__ bool mbar_test_wait(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
 constexpr uint32_t WAIT_POLLS = 1u << 20;  // each poll suspends for at most ~2 us: a wait gives up after about 2 s
 
 // Waits for the phase with the given parity to complete.  Returns false if it gave up, either
 // because the poll budget ran out (it then raises *abort_flag) or because another thread of the
 // CTA raised *abort_flag.
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
+    if (mbar_test_wait(bar, parity)) return true;   // the common case in a pipeline that runs ahead
     for (uint32_t it = 0; it < WAIT_POLLS; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 63u) == 63u && *abort_flag) return false;
-        if (it >= 2) __nanosleep(it < 16 ? 64 : 256);   // back off: a spinning warp steals issue slots from working ones
+        if (it >= 64) __nanosleep(64);   // a long wait backs off; a hand-over between pipeline stages must not oversleep
     }
     *abort_flag = 1;
     return false;
