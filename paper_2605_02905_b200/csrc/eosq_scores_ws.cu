@@ -103,7 +103,7 @@ __device__ __forceinline__ void ws_split_store(uint8_t *plane, int g, int k, flo
 
 struct WsBarriers {
     uint64_t st_full[WS_STAGES], st_empty[WS_STAGES];
-    uint64_t a_full[WS_BUFS], a_empty[WS_BUFS], d_full[WS_BUFS], d_empty[WS_BUFS];
+    uint64_t a_full[WS_BUFS], d_full[WS_BUFS], d_empty[WS_BUFS];
     uint64_t blk_full[2], blk_empty[2], b2_full[2], b2_empty[2], b1_full[2], b1_empty[2];
 };
 
@@ -130,7 +130,6 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
         }
         for (int b = 0; b < WS_BUFS; ++b) {
             mbar_init(&bars.a_full[b], 4);             // one arrival per warp: 128 arrivals on one barrier serialise
-            mbar_init(&bars.a_empty[b], 1);
             mbar_init(&bars.d_full[b], 1);
             mbar_init(&bars.d_empty[b], 4);
         }
@@ -240,7 +239,8 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
                 for (int tile = 0; tile < tiles; ++tile, ++seq) {
                     const int buf = seq & (WS_BUFS - 1);
                     const uint32_t u = (seq >> 2) & 1u;
-                    if (!mbar_wait(&bars.a_full[buf], u, &abort_flag) || !mbar_wait(&bars.d_empty[buf], u ^ 1u, &abort_flag)) {
+                    // a filled buffer is also a drained one: its expanders waited for the epilogue of its last use
+                    if (!mbar_wait(&bars.a_full[buf], u, &abort_flag)) {
                         alive = false;
                         break;
                     }
@@ -249,8 +249,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
 #pragma unroll
                     for (int ks = 0; ks < D / 16; ++ks) umma_f16_ts(tb + WS_COL_D1, tb + 8 * ks, bdesc[ks], idesc, ks ? 1u : 0u);
                     umma_f16_ts(tb + WS_COL_D2, tb + WS_COL_P, bdesc[D / 16], idesc, 0u);
-                    umma_commit(&bars.d_full[buf]);
-                    umma_commit(&bars.a_empty[buf]);
+                    umma_commit(&bars.d_full[buf]);   // the one commit of a tile: each costs the issuing thread well over 100 cycles
                 }
                 if (!alive) break;
                 umma_commit(&bars.b2_empty[vb]);
@@ -416,7 +415,8 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
                     for (int i = 0; i < 8; ++i) pw[i] = 0u;
                 }
                 const uint32_t u = (seq >> 2) & 1u;
-                if (!mbar_wait(&bars.a_empty[buf], u ^ 1u, &abort_flag) || !mbar_wait(&bars.d_empty[buf], u ^ 1u, &abort_flag)) {
+                // the epilogue has read the last use of this buffer, hence its MMAs are over too
+                if (!mbar_wait(&bars.d_empty[buf], u ^ 1u, &abort_flag)) {
                     alive = false;
                     break;
                 }
