@@ -259,7 +259,8 @@ def run_library(args):
     achieved = units * blocks_per_launch / (dom_ms_per_launch * 1e-3)
     # DRAM bytes per block from the committed ncu section capture (profiles/sections_per_kernel_*.txt),
     # scaled to the blocks of one launch; None for kernels changed since that capture
-    ncu_traffic_per_block = {"gram": 186e6 / 592}
+    ncu_traffic_per_block = {"gram": 187.4e6 / 592, "tridiag_a": 86.4e6 / 592, "tridiag_b": 44.4e6 / 592, "tridiag_c": 20.1e6 / 592,
+                             "eigvals": 1.2e6 / 592, "spectral": 81.6e6 / 592, "quant": 177.9e6 / 592}
     traffic = ncu_traffic_per_block.get(dominant)
     roofline = {"kernel": dominant, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit,
                 "frac": achieved / peak, "traffic": (traffic * blocks_per_launch if traffic else None),
