@@ -337,10 +337,13 @@ __global__ void __launch_bounds__(QT_THREADS, 2) quant_tc_kernel(const __grid_co
     for (int b = blockIdx.x; b < nb && !abort_flag; b += gridDim.x) {
         const int rank = ws.rank[b];
         // ---- B = [M | coef V], split and swizzled ---------------------------------------------
-        for (int e = tid; e < RMAX * D; e += QT_THREADS) Vc[e] = ws.vr[static_cast<size_t>(b) * RMAX * D + e];
-        __syncthreads();
-        {   // W[i][c] = sum_j Pi[c][j] zeta_i[j]
+        {   // W[i][c] = sum_j Pi[c][j] zeta_i[j]; the rotation comes from L2, a batch of 32 rows ahead of its use
             const int c = tid & (D - 1), half = tid >> 7;
+            float pn[32];
+#pragma unroll
+            for (int jj = 0; jj < 32; ++jj) pn[jj] = __ldg(pi_t + jj * D + c);
+            for (int e = tid; e < RMAX * D; e += QT_THREADS) Vc[e] = ws.vr[static_cast<size_t>(b) * RMAX * D + e];
+            __syncthreads();
             float w[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) w[i] = 0.0f;
@@ -349,7 +352,11 @@ __global__ void __launch_bounds__(QT_THREADS, 2) quant_tc_kernel(const __grid_co
                 for (int j0 = 0; j0 < D; j0 += 32) {
                     float pv[32];
 #pragma unroll
-                    for (int jj = 0; jj < 32; ++jj) pv[jj] = __ldg(pi_t + (j0 + jj) * D + c);   // 32 loads in flight
+                    for (int jj = 0; jj < 32; ++jj) pv[jj] = pn[jj];
+                    if (j0 + 32 < D) {
+#pragma unroll
+                        for (int jj = 0; jj < 32; ++jj) pn[jj] = __ldg(pi_t + (j0 + 32 + jj) * D + c);
+                    }
 #pragma unroll
                     for (int jj = 0; jj < 32; jj += 4) {
 #pragma unroll
@@ -369,11 +376,17 @@ __global__ void __launch_bounds__(QT_THREADS, 2) quant_tc_kernel(const __grid_co
         __syncthreads();
         for (int e = tid; e < RMAX * D; e += QT_THREADS) Vc[e] *= ws.coef[static_cast<size_t>(b) * RMAX + e / D];
         __syncthreads();
+        // chunk = 8 consecutive entries of a row of M; a thread's chunks are QT_THREADS apart, i.e. 16 rows,
+        // and the rotation entries of the next chunk are fetched while the current one is worked on
+        float4 n0 = __ldg(reinterpret_cast<const float4 *>(pi + tid * 8)), n1 = __ldg(reinterpret_cast<const float4 *>(pi + tid * 8 + 4));
 #pragma unroll 1
         for (int it = 0; it < (D * D / 8) / QT_THREADS; ++it) {
             const int chunk = tid + QT_THREADS * it, c = chunk >> 4, jc = chunk & 15;
-            const float4 p0 = *reinterpret_cast<const float4 *>(pi + c * D + 8 * jc);
-            const float4 p1 = *reinterpret_cast<const float4 *>(pi + c * D + 8 * jc + 4);
+            const float4 p0 = n0, p1 = n1;
+            if (it + 1 < (D * D / 8) / QT_THREADS) {
+                n0 = __ldg(reinterpret_cast<const float4 *>(pi + (chunk + QT_THREADS) * 8));
+                n1 = __ldg(reinterpret_cast<const float4 *>(pi + (chunk + QT_THREADS) * 8 + 4));
+            }
             float m[8] = {p0.x, p0.y, p0.z, p0.w, p1.x, p1.y, p1.z, p1.w};
             for (int i = 0; i < rank; ++i) {
                 const float w = W[i * D + c];
