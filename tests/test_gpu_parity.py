@@ -146,6 +146,22 @@ def test_many_blocks_cross_the_chunk_boundary_and_are_deterministic(ctx):
     _report("chunks", rep)
 
 
+def test_profile_select_times_only_the_chosen_stage(ctx):
+    """eosq_profile_select brackets the launches of the named stages only; the count of all launches goes on."""
+    w = synth.kv_cache_blocks("prof", layers=1, kv_heads=2, tokens=512, n=256, rank_hi=4, seed=61)
+    n0 = ctx.launch_count
+    ctx.profile_select(["quant", "tridiag_b"])
+    try:
+        _encode(ctx, w.blocks, 2)
+        stages = ctx.profile_read()
+    finally:
+        ctx.profile_enable(False)
+    timed = {k for k, v in stages.items() if v[1]}
+    assert timed == {"quant", "tridiag_b"}, timed
+    assert stages["quant"][0] > 0.0 and stages["quant"][1] == 1
+    assert ctx.launch_count - n0 >= 12   # Gram, three tridiagonalisation ranges, eigenvalues, second pass, spectral, quantise
+
+
 def test_host_buffer_entry_point_matches_device_path(ctx):
     w = synth.kv_cache_blocks("host", layers=1, kv_heads=2, tokens=512, n=256, rank_hi=6, seed=60)
     dev, cache = _encode(ctx, w.blocks, 2)
