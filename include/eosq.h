@@ -185,7 +185,10 @@ int eosq_scores(eosq_ctx *ctx, const eosq_cache_t *kcache, int64_t num_kv_heads,
  * Host-buffer convenience for end-to-end use: copies `blocks` (host, pinned preferred) to the
  * device in chunks, encodes, and copies codes, norms, rank, sigma, phi, P, V and status back into
  * the host arrays of `host_out` (optional members may be null).  `arena` is dev scratch of at least
- * eosq_encode_host_arena_bytes().  Synchronises the stream before returning.
+ * eosq_encode_host_arena_bytes(): two slots of one chunk's input and outputs plus one workspace.
+ * Uploads and downloads run on two streams the context owns, the kernels on `cuda_stream`, so that
+ * with pinned host memory the three overlap; work already queued on `cuda_stream` is waited for
+ * first.  Synchronises all three streams before returning.
  */
 size_t eosq_encode_host_arena_bytes(int64_t num_blocks, int n, int d, int bits, int in_dtype);
 int eosq_encode_host(eosq_ctx *ctx, const void *host_blocks, int in_dtype, int64_t num_blocks, int n,

@@ -197,6 +197,14 @@ extern "C" int eosq_destroy(eosq_ctx *ctx) {
         cudaEventDestroy(t.stop);
     }
     for (cudaEvent_t e : ctx->free_events) cudaEventDestroy(e);
+    if (ctx->copy_in) cudaStreamDestroy(ctx->copy_in);
+    if (ctx->copy_out) cudaStreamDestroy(ctx->copy_out);
+    if (ctx->ev_start) cudaEventDestroy(ctx->ev_start);
+    for (int i = 0; i < 2; ++i) {
+        if (ctx->ev_in[i]) cudaEventDestroy(ctx->ev_in[i]);
+        if (ctx->ev_done[i]) cudaEventDestroy(ctx->ev_done[i]);
+        if (ctx->ev_out[i]) cudaEventDestroy(ctx->ev_out[i]);
+    }
     delete ctx;
     return EOSQ_OK;
 }
@@ -325,9 +333,13 @@ extern "C" int eosq_scores(eosq_ctx *ctx, const eosq_cache_t *kcache, int64_t nu
 namespace {
 constexpr int64_t HOST_CHUNK = 1184;
 
+// Two slots (input chunk + its outputs) so that the upload of chunk i + 1 and the download of chunk
+// i - 1 run while chunk i is encoded, and one workspace (encodes run one after another).
+constexpr int HOST_SLOTS = 2;
+
 struct Arena {
-    void *in;
-    eosq_cache_t dev;
+    void *in[HOST_SLOTS];
+    eosq_cache_t dev[HOST_SLOTS];
     void *ws;
     size_t ws_bytes;
 };
@@ -343,21 +355,38 @@ size_t carve_arena(void *base, int64_t cap, int n, int bits, int in_dtype, Arena
     Arena r;
     std::memset(&r, 0, sizeof(r));
     const size_t esize = (in_dtype == EOSQ_F32) ? 4 : 2;
-    r.in = take(static_cast<size_t>(cap) * n * D * esize);
-    r.dev.codes = static_cast<uint8_t *>(take(static_cast<size_t>(cap) * n * D * bits / 8));
-    r.dev.norms = static_cast<uint16_t *>(take(static_cast<size_t>(cap) * n * 2));
-    r.dev.rank = static_cast<int32_t *>(take(static_cast<size_t>(cap) * 4));
-    r.dev.sigma = static_cast<float *>(take(static_cast<size_t>(cap) * RMAX * 4));
-    r.dev.phi = static_cast<float *>(take(static_cast<size_t>(cap) * RMAX * 4));
-    r.dev.P = static_cast<uint16_t *>(take(static_cast<size_t>(cap) * RMAX * n * 2));
-    r.dev.V = static_cast<uint16_t *>(take(static_cast<size_t>(cap) * RMAX * D * 2));
-    r.dev.status = static_cast<int32_t *>(take(static_cast<size_t>(cap) * 4));
-    r.dev.eig = static_cast<float *>(take(static_cast<size_t>(cap) * D * 4));
-    r.dev.lambda_plus = static_cast<float *>(take(static_cast<size_t>(cap) * 4));
+    for (int slot = 0; slot < HOST_SLOTS; ++slot) {
+        eosq_cache_t &c = r.dev[slot];
+        r.in[slot] = take(static_cast<size_t>(cap) * n * D * esize);
+        c.codes = static_cast<uint8_t *>(take(static_cast<size_t>(cap) * n * D * bits / 8));
+        c.norms = static_cast<uint16_t *>(take(static_cast<size_t>(cap) * n * 2));
+        c.rank = static_cast<int32_t *>(take(static_cast<size_t>(cap) * 4));
+        c.sigma = static_cast<float *>(take(static_cast<size_t>(cap) * RMAX * 4));
+        c.phi = static_cast<float *>(take(static_cast<size_t>(cap) * RMAX * 4));
+        c.P = static_cast<uint16_t *>(take(static_cast<size_t>(cap) * RMAX * n * 2));
+        c.V = static_cast<uint16_t *>(take(static_cast<size_t>(cap) * RMAX * D * 2));
+        c.status = static_cast<int32_t *>(take(static_cast<size_t>(cap) * 4));
+        c.eig = static_cast<float *>(take(static_cast<size_t>(cap) * D * 4));
+        c.lambda_plus = static_cast<float *>(take(static_cast<size_t>(cap) * 4));
+    }
     r.ws_bytes = eosq_workspace_bytes(cap, n, D);
     r.ws = take(r.ws_bytes);
     if (a) *a = r;
     return off;
+}
+
+// Streams and events of the host-buffer path, made once per context.
+bool host_path_ready(eosq_ctx *ctx) {
+    if (ctx->copy_in) return true;
+    cudaError_t e = cudaStreamCreateWithFlags(&ctx->copy_in, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->copy_out, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_start, cudaEventDisableTiming);
+    for (int i = 0; i < HOST_SLOTS && e == cudaSuccess; ++i) {
+        e = cudaEventCreateWithFlags(&ctx->ev_in[i], cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_done[i], cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_out[i], cudaEventDisableTiming);
+    }
+    return !record_cuda(ctx, e, "host path streams and events");
 }
 }  // namespace
 
@@ -376,26 +405,45 @@ extern "C" int eosq_encode_host(eosq_ctx *ctx, const void *host_blocks, int in_d
     if (!host_blocks || !cache_required_ok(host_out) || !arena || (reinterpret_cast<uintptr_t>(arena) & 255u))
         return EOSQ_ERR_INVALID_ARG;
     if (arena_bytes < eosq_encode_host_arena_bytes(num_blocks, n, d, bits, in_dtype)) return EOSQ_ERR_BUFFER_TOO_SMALL;
-    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    if (!host_path_ready(ctx)) return EOSQ_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream), s_in = ctx->copy_in, s_out = ctx->copy_out;
     const int64_t cap = std::min<int64_t>(num_blocks, HOST_CHUNK);
     Arena a;
     carve_arena(arena, cap, n, bits, in_dtype, &a);
     const size_t esize = (in_dtype == EOSQ_F32) ? 4 : 2;
     const size_t rb = static_cast<size_t>(D) * bits / 8;
-    for (int64_t b0 = 0; b0 < num_blocks; b0 += cap) {
+    cudaError_t e = cudaSuccess;
+    auto ok = [&](cudaError_t r) {
+        if (e == cudaSuccess) e = r;
+        return e == cudaSuccess;
+    };
+    // Three streams: uploads, the caller's stream for the kernels, downloads.  Slot i % 2 is handed
+    // round by events: uploaded -> encoded -> downloaded -> free for the upload of chunk i + 2.
+    // Whatever the caller's stream still does with the arena comes first.
+    ok(cudaEventRecord(ctx->ev_start, s));
+    ok(cudaStreamWaitEvent(s_in, ctx->ev_start, 0));
+    ok(cudaStreamWaitEvent(s_out, ctx->ev_start, 0));
+    int64_t chunk = 0;
+    for (int64_t b0 = 0; b0 < num_blocks && e == cudaSuccess; b0 += cap, ++chunk) {
+        const int slot = static_cast<int>(chunk % HOST_SLOTS);
         const int64_t nb = std::min<int64_t>(cap, num_blocks - b0);
         const char *src = static_cast<const char *>(host_blocks) + static_cast<size_t>(b0) * n * D * esize;
-        if (record_cuda(ctx, cudaMemcpyAsync(a.in, src, static_cast<size_t>(nb) * n * D * esize, cudaMemcpyHostToDevice, s), "h2d"))
-            return EOSQ_ERR_CUDA;
-        eosq_cache_t dev = a.dev;
+        if (chunk >= HOST_SLOTS) ok(cudaStreamWaitEvent(s_in, ctx->ev_done[slot], 0));   // the slot's last encode has read its input
+        ok(cudaMemcpyAsync(a.in[slot], src, static_cast<size_t>(nb) * n * D * esize, cudaMemcpyHostToDevice, s_in));
+        ok(cudaEventRecord(ctx->ev_in[slot], s_in));
+        ok(cudaStreamWaitEvent(s, ctx->ev_in[slot], 0));
+        if (chunk >= HOST_SLOTS) ok(cudaStreamWaitEvent(s, ctx->ev_out[slot], 0));       // the slot's last outputs are on the host
+        if (e != cudaSuccess) break;
+        eosq_cache_t dev = a.dev[slot];
         if (!host_out->eig) dev.eig = nullptr;
         if (!host_out->lambda_plus) dev.lambda_plus = nullptr;
-        rc = eosq_encode(ctx, a.in, in_dtype, nb, n, d, bits, seed, &dev, a.ws, a.ws_bytes, s);
-        if (rc != EOSQ_OK) return rc;
+        rc = eosq_encode(ctx, a.in[slot], in_dtype, nb, n, d, bits, seed, &dev, a.ws, a.ws_bytes, s);
+        if (rc != EOSQ_OK) break;
+        ok(cudaEventRecord(ctx->ev_done[slot], s));
+        ok(cudaStreamWaitEvent(s_out, ctx->ev_done[slot], 0));
         const eosq_cache_t h = shifted(*host_out, b0, n, bits);
-        cudaError_t e = cudaSuccess;
         auto back = [&](void *dst, const void *srcp, size_t bytes) {
-            if (e == cudaSuccess && dst) e = cudaMemcpyAsync(dst, srcp, bytes, cudaMemcpyDeviceToHost, s);
+            if (dst) ok(cudaMemcpyAsync(dst, srcp, bytes, cudaMemcpyDeviceToHost, s_out));
         };
         back(h.codes, dev.codes, static_cast<size_t>(nb) * n * rb);
         back(h.norms, dev.norms, static_cast<size_t>(nb) * n * 2);
@@ -407,9 +455,16 @@ extern "C" int eosq_encode_host(eosq_ctx *ctx, const void *host_blocks, int in_d
         back(h.status, dev.status, static_cast<size_t>(nb) * 4);
         if (dev.eig) back(h.eig, dev.eig, static_cast<size_t>(nb) * D * 4);
         if (dev.lambda_plus) back(h.lambda_plus, dev.lambda_plus, static_cast<size_t>(nb) * 4);
-        if (record_cuda(ctx, e, "d2h")) return EOSQ_ERR_CUDA;
+        ok(cudaEventRecord(ctx->ev_out[slot], s_out));
     }
-    if (record_cuda(ctx, cudaStreamSynchronize(s), "cudaStreamSynchronize")) return EOSQ_ERR_CUDA;
+    // Everything this call enqueued is waited for, also after an error: the caller owns the arena again.
+    cudaStreamSynchronize(s_in);
+    const cudaError_t e1 = cudaStreamSynchronize(s);
+    const cudaError_t e2 = cudaStreamSynchronize(s_out);
+    if (rc != EOSQ_OK) return rc;
+    if (record_cuda(ctx, e, "host path copy or event")) return EOSQ_ERR_CUDA;
+    if (record_cuda(ctx, e1, "cudaStreamSynchronize")) return EOSQ_ERR_CUDA;
+    if (record_cuda(ctx, e2, "cudaStreamSynchronize(download stream)")) return EOSQ_ERR_CUDA;
     return EOSQ_OK;
 }
 

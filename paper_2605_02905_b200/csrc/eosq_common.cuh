@@ -99,6 +99,9 @@ struct eosq_ctx {
     uint32_t profile_mask = 0;   // bit i set: launches of stage i are bracketed by events
     std::vector<Timed> timed;
     std::vector<cudaEvent_t> free_events;
+    // host-buffer path: copy streams and hand-over events of its two arena slots (created on first use)
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;
+    cudaEvent_t ev_start = nullptr, ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
 };
 
 namespace eosq {
