@@ -277,6 +277,28 @@ def run_library(args):
     scores_roofline = {"bound": "hbm", "achieved": sc_gbs / world, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                        "frac": (t_sc_roof * 1e3 / sc_ms) if k_blocks else None}
 
+    # ---- decode (Algorithm 1 DeQuant + low-rank part), timed on its own: it is not part of a step ----
+    decode = None
+    if not args.no_decode:
+        dec_out = torch.empty((B, n, d), dtype=torch.float16, device="cuda")
+        for _ in range(2):
+            eosq.eosq_decode(ctx, cache, SEED, out=dec_out)
+        torch.cuda.synchronize()
+        reps = max(2, min(args.steps, 5))
+        d0 = torch.cuda.Event(enable_timing=True)
+        d1 = torch.cuda.Event(enable_timing=True)
+        d0.record()
+        for _ in range(reps):
+            eosq.eosq_decode(ctx, cache, SEED, out=dec_out)
+        d1.record()
+        torch.cuda.synchronize()
+        dec_ms = shard.max_over_ranks([d0.elapsed_time(d1) / reps], device="cuda")[0]
+        dec_bytes = B * n * d * 2 + B * out_bytes_per_block   # fp16 out + compressed in
+        decode = {"ms": dec_ms, "gbs": world * dec_bytes / (dec_ms * 1e-3) / 1e9, "bytes": dec_bytes,
+                  "roofline": {"bound": "hbm", "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                               "frac": dec_bytes / (dec_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}}
+        del dec_out
+
     # ---- end to end through the host-buffer entry point ------------------------------------------
     e2e = None
     cpu_baseline = None
@@ -326,6 +348,7 @@ def run_library(args):
                        "flagged_blocks": flagged},
             "encode": {"ms": enc_ms, "gbs_in": enc_gbs},
             "scores": {"ms": sc_ms, "gbs_compressed": sc_gbs, "bytes": score_bytes, "roofline": scores_roofline},
+            "decode": decode,
             "roofline": roofline, "encode_roofline": encode_roofline,
             "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": launches, "clocks": clocks.summary(),
         }
@@ -344,6 +367,7 @@ def main():
     ap.add_argument("--blocks", type=int, default=None, help="encode only the first BLOCKS blocks (profiling captures)")
     ap.add_argument("--e2e-blocks", type=int, default=None, help="blocks per end-to-end host-buffer call (default: the whole cache)")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-decode", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -288,7 +288,16 @@ extern "C" int eosq_decode(eosq_ctx *ctx, const eosq_cache_t *cache, int64_t num
     if ((rc = get_rotation(ctx, d, seed, &rot)) != EOSQ_OK) return rc;
     if ((rc = get_codebook(d, bits, &cb)) != EOSQ_OK) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    run_stage(ctx, ST_DECODE, s, [&] { launch_decode_plain(*cache, num_blocks, n, rot, cb, out_blocks, out_dtype, s); });
+    if (decode_tc_supported(*cache, bits, out_blocks)) {
+        bool setup_ok = true;
+        run_stage(ctx, ST_DECODE, s, [&] { setup_ok = launch_decode_tc(*cache, num_blocks, n, rot, cb, out_blocks, out_dtype, ctx->dev_err, ctx->sm_count, s); });
+        if (!setup_ok) {
+            ctx->last_error = "tensor-core decode kernel: launch set-up failed";
+            return EOSQ_ERR_CUDA;
+        }
+    } else {
+        run_stage(ctx, ST_DECODE, s, [&] { launch_decode_plain(*cache, num_blocks, n, rot, cb, out_blocks, out_dtype, s); });
+    }
     if (record_cuda(ctx, cudaGetLastError(), "eosq_decode launch")) return EOSQ_ERR_CUDA;
     return EOSQ_OK;
 }

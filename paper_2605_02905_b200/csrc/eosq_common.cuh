@@ -146,6 +146,9 @@ bool launch_quant_tc(const void *blocks_all, int64_t block0, int64_t nb, int n, 
                      const Codebook &cb, const eosq_cache_t &out, int *err, int sm_count, cudaStream_t s);
 void launch_decode_plain(const eosq_cache_t &cache, int64_t nb, int n, const Rotation &rot, const Codebook &cb,
                          void *out_blocks, int out_dtype, cudaStream_t s);
+bool decode_tc_supported(const eosq_cache_t &cache, int bits, const void *out_blocks);
+bool launch_decode_tc(const eosq_cache_t &cache, int64_t nb, int n, const Rotation &rot, const Codebook &cb, void *out_blocks,
+                      int out_dtype, int *err, int sm_count, cudaStream_t s);
 void launch_scores_plain(const eosq_cache_t &cache, int64_t heads, int64_t bph, int64_t head_stride, int n,
                          const Rotation &rot, const Codebook &cb, const __half *q, int G, float scale,
                          float *scores, cudaStream_t s);

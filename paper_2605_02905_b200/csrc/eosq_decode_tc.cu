@@ -1,0 +1,285 @@
+// Tensor-core decode for 2-bit codes (Algorithm 1 DeQuant + the stored low-rank part):
+//   x_t = rho_t (z_t Pi) + sum_i P[t][i] zeta_i,     z_t = centroids of the codes of token t.
+//
+// One persistent CTA of 512 threads per SM holds the rotation once, as the B operand of
+//   D1[128 tokens][128] = Z[128][128] (fp16 centroids) x Pi      (Pi scaled by 2^12 and split
+//                                                                  into a high and a low fp16 plane),
+//   D2[128 tokens][128] = P_tile[128][16] x V[16][128]            (stored fp16 factors: exact products),
+// both accumulated in fp32 in tensor memory.  The two halves of the CTA (256 threads each) work
+// on different blocks like two CTAs would - each with its own operand buffers, half of the tensor
+// memory and its own barriers - so that one half's MMAs overlap the other's expansion and stores.
+// Per 128-token tile a half expands the codes into a K-major 128-byte-swizzled A tile (byte
+// permutes), writes the factor rows next to it, one thread issues the 17 MMAs, and every thread
+// turns 64 columns of one token's accumulators into rho D1 / (kappa 2^12) + D2 and stores them.
+#include <algorithm>
+#include <cstdint>
+
+#include "eosq_common.cuh"
+#include "eosq_expand.cuh"
+#include "eosq_sm100.cuh"
+
+namespace eosq {
+
+using namespace sm100;
+
+constexpr int TC_ERR_DECODE_TIMEOUT = 16;
+
+constexpr int DT_THREADS = 512, DT_HALF = 256;
+constexpr float DT_PSCALE = 4096.0f;                  // keeps the low plane of Pi in fp16's normal range
+constexpr uint32_t DT_BOX = 128 * 128;                // 128 rows x 64 fp16 of K
+constexpr uint32_t DT_OFF_PI_HI = 0, DT_OFF_PI_LO = 2 * DT_BOX;
+constexpr uint32_t DT_OFF_HALF = 4 * DT_BOX;          // per half: A tile (2 boxes), factor tile (1 box), right vectors (1 box)
+constexpr uint32_t DT_HALF_BYTES = 4 * DT_BOX;
+constexpr uint32_t DT_H_A = 0, DT_H_P = 2 * DT_BOX, DT_H_V = 3 * DT_BOX;
+constexpr size_t DT_SMEM = DT_OFF_HALF + 2 * DT_HALF_BYTES + 1024;   // 193 KB
+constexpr uint32_t DT_TMEM_COLS = 512;                // per half: D1 128 columns, D2 128 columns
+
+// Byte offset of the 16-byte chunk `jc` (8 fp16 of K) of row `row` in a K-major, 128-byte-swizzled
+// operand of 128 rows: 64-wide K boxes of 16 KB, 8-row groups of 1 KB, chunks XOR-ed with the row.
+__device__ __forceinline__ uint32_t dt_offset(int row, int jc) {
+    return (jc >> 3) * DT_BOX + (row >> 3) * 1024 + (row & 7) * 128 + (((jc & 7) ^ (row & 7)) << 4);
+}
+
+__device__ __forceinline__ void dt_bar_sync(int half) {
+    asm volatile("bar.sync %0, %1;" ::"r"(1 + half), "r"(DT_HALF) : "memory");
+}
+
+struct DecodeArgs {
+    eosq_cache_t cache;
+    int nb, n;
+    float inv_scale;            // 1 / (kappa 2^12)
+    uint32_t lo_tab, hi_tab;    // bytes of the four fp16 centroids times kappa
+    const float *pi_t;          // pi_t[j][c] = Pi[c][j]
+    void *out;
+    int *err;
+};
+
+// What a thread fetches from global memory for one tile: 64 codes of its token, the token's norm,
+// and (threads of the first column half only) the token's factor entries, packed.
+struct DtTileRegs {
+    uint4 codes;
+    uint4 p0, p1;
+    float rho;
+};
+
+template <typename Tout>
+__global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeArgs a) {
+    extern __shared__ uint8_t dt_smem_raw[];
+    __shared__ __align__(8) uint64_t mma_done[2];
+    __shared__ uint32_t tmem_base_s;
+    __shared__ volatile int abort_flag;
+
+    uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(dt_smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int half = tid >> 8, ht = tid & (DT_HALF - 1);
+    const int r = ht & 127, box = ht >> 7;   // token within the tile (= tensor-memory lane), column half
+    const int n = a.n, tiles = (n + 127) / 128;
+
+    if (tid == 0) {
+        mbar_init(&mma_done[0], 1);
+        mbar_init(&mma_done[1], 1);
+        abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 0) {
+        tmem_alloc(&tmem_base_s, DT_TMEM_COLS);
+        tmem_relinquish();
+    }
+    // B operand of D1, once per CTA: row j (output coordinate), K = c: Pi[c][j] 2^12 as high + low fp16
+    for (int chunk = tid; chunk < D * (D / 8); chunk += DT_THREADS) {
+        const int j = chunk >> 4, jc = chunk & 15;
+        const float4 p0 = __ldg(reinterpret_cast<const float4 *>(a.pi_t + j * D + 8 * jc));
+        const float4 p1 = __ldg(reinterpret_cast<const float4 *>(a.pi_t + j * D + 8 * jc + 4));
+        const float m[8] = {p0.x, p0.y, p0.z, p0.w, p1.x, p1.y, p1.z, p1.w};
+        uint32_t h[4], l[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float x0 = m[2 * e] * DT_PSCALE, x1 = m[2 * e + 1] * DT_PSCALE;
+            const __half h0 = __float2half_rn(x0), h1 = __float2half_rn(x1);
+            const __half l0 = __float2half_rn(x0 - __half2float(h0)), l1 = __float2half_rn(x1 - __half2float(h1));
+            h[e] = static_cast<uint32_t>(__half_as_ushort(h0)) | (static_cast<uint32_t>(__half_as_ushort(h1)) << 16);
+            l[e] = static_cast<uint32_t>(__half_as_ushort(l0)) | (static_cast<uint32_t>(__half_as_ushort(l1)) << 16);
+        }
+        const uint32_t off = dt_offset(j, jc);
+        *reinterpret_cast<uint4 *>(base + DT_OFF_PI_HI + off) = make_uint4(h[0], h[1], h[2], h[3]);
+        *reinterpret_cast<uint4 *>(base + DT_OFF_PI_LO + off) = make_uint4(l[0], l[1], l[2], l[3]);
+    }
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+
+    uint8_t *hbase = base + DT_OFF_HALF + half * DT_HALF_BYTES;
+    const uint32_t d1 = tmem_base_s + 256u * half, d2 = d1 + 128u;
+    const uint32_t lane_off = static_cast<uint32_t>(32 * (warp & 3)) << 16;   // a warp reaches lanes 32 (warp % 4)..
+    const uint16_t *Pg = a.cache.P;
+    Tout *outp = static_cast<Tout *>(a.out);
+
+    auto fetch = [&](long long blk, int tile, int rank) {
+        DtTileRegs g;
+        const int tok = tile * 128 + r;
+        const bool valid = tok < n;
+        const size_t t = static_cast<size_t>(blk) * n + tok;
+        g.codes = valid ? __ldg(reinterpret_cast<const uint4 *>(a.cache.codes + t * 32 + 16 * box)) : make_uint4(0u, 0u, 0u, 0u);
+        g.rho = valid ? __half2float(__ushort_as_half(a.cache.norms[t])) : 0.0f;
+        uint32_t pw[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) pw[i] = 0u;
+        if (box == 0 && valid) {
+#pragma unroll
+            for (int i = 0; i < RMAX; ++i) {
+                if (i < rank) {
+                    const uint32_t v = Pg[(static_cast<size_t>(blk) * RMAX + i) * n + tok];
+                    pw[i >> 1] |= v << (16 * (i & 1));
+                }
+            }
+        }
+        g.p0 = make_uint4(pw[0], pw[1], pw[2], pw[3]);
+        g.p1 = make_uint4(pw[4], pw[5], pw[6], pw[7]);
+        return g;
+    };
+
+    uint32_t phase = 0;
+    bool alive = true;
+    for (long long blk = 2ll * blockIdx.x + half; blk < a.nb && alive; blk += 2ll * gridDim.x) {
+        const int rank = max(0, min(a.cache.rank[blk], RMAX));
+        {   // B operand of D2: row j, K = i: zeta_i[j] (zero beyond the rank); this thread: row r, entries 8 box .. 8 box + 7
+            uint32_t vw[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const int i = 8 * box + e;
+                if (i < rank) vw[e >> 1] |= static_cast<uint32_t>(a.cache.V[(static_cast<size_t>(blk) * RMAX + i) * D + r]) << (16 * (e & 1));
+            }
+            *reinterpret_cast<uint4 *>(hbase + DT_H_V + dt_offset(r, box)) = make_uint4(vw[0], vw[1], vw[2], vw[3]);
+        }
+        DtTileRegs g = fetch(blk, 0, rank);
+        for (int tile = 0; tile < tiles; ++tile) {
+            {   // A operand of D1: this token's 64 coordinates of column half `box`, as fp16 centroids
+                const uint32_t w[4] = {g.codes.x, g.codes.y, g.codes.z, g.codes.w};
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    uint32_t o[8];
+                    expand16_2bit(w[q], a.lo_tab, a.hi_tab, o);
+                    *reinterpret_cast<uint4 *>(hbase + DT_H_A + dt_offset(r, 8 * box + 2 * q)) = make_uint4(o[0], o[1], o[2], o[3]);
+                    *reinterpret_cast<uint4 *>(hbase + DT_H_A + dt_offset(r, 8 * box + 2 * q + 1)) = make_uint4(o[4], o[5], o[6], o[7]);
+                }
+                if (box == 0) {   // A operand of D2: the token's factor entries
+                    *reinterpret_cast<uint4 *>(hbase + DT_H_P + dt_offset(r, 0)) = g.p0;
+                    *reinterpret_cast<uint4 *>(hbase + DT_H_P + dt_offset(r, 1)) = g.p1;
+                }
+            }
+            const float f = g.rho * a.inv_scale;
+            fence_proxy_async_smem();   // the operands were written by ordinary stores and are read by the tensor core
+            dt_bar_sync(half);
+            if (ht == 0) {
+                tc_fence_after_sync();
+                constexpr uint32_t idesc = umma_idesc_f16(128, D, false, false);
+                const uint32_t a0 = smem_u32(hbase + DT_H_A), hi0 = smem_u32(base + DT_OFF_PI_HI), lo0 = smem_u32(base + DT_OFF_PI_LO);
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    const uint32_t ko = (ks >> 2) * DT_BOX + (ks & 3) * 32;
+                    const uint64_t da = umma_desc_sw128(a0 + ko, 16, 1024);
+                    umma_f16(d1, da, umma_desc_sw128(hi0 + ko, 16, 1024), idesc, ks ? 1u : 0u);
+                    umma_f16(d1, da, umma_desc_sw128(lo0 + ko, 16, 1024), idesc, 1u);
+                }
+                umma_f16(d2, umma_desc_sw128(smem_u32(hbase + DT_H_P), 16, 1024), umma_desc_sw128(smem_u32(hbase + DT_H_V), 16, 1024), idesc, 0u);
+                umma_commit(&mma_done[half]);
+            }
+            if (tile + 1 < tiles) g = fetch(blk, tile + 1, rank);   // behind the MMAs
+            if (!mbar_wait(&mma_done[half], phase, &abort_flag)) {
+                alive = false;
+                break;
+            }
+            phase ^= 1u;
+            tc_fence_after_sync();
+            const int tok = tile * 128 + r;
+            Tout *dst = outp + (static_cast<size_t>(blk) * n + tok) * D + 64 * box;
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                uint32_t v1[32], v2[32];
+                tmem_ld32(d1 + lane_off + 64u * box + 32u * c, v1);
+                tmem_ld32(d2 + lane_off + 64u * box + 32u * c, v2);
+                tmem_ld_wait();
+                if (tok < n) {
+                    if (sizeof(Tout) == 2) {
+                        uint32_t pk[16];
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) {
+                            const float x0 = fmaf(f, __uint_as_float(v1[2 * e]), __uint_as_float(v2[2 * e]));
+                            const float x1 = fmaf(f, __uint_as_float(v1[2 * e + 1]), __uint_as_float(v2[2 * e + 1]));
+                            pk[e] = static_cast<uint32_t>(__half_as_ushort(__float2half_rn(x0))) |
+                                    (static_cast<uint32_t>(__half_as_ushort(__float2half_rn(x1))) << 16);
+                        }
+                        uint4 *d4 = reinterpret_cast<uint4 *>(dst + 32 * c);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) d4[e] = make_uint4(pk[4 * e], pk[4 * e + 1], pk[4 * e + 2], pk[4 * e + 3]);
+                    } else {
+                        float4 *d4 = reinterpret_cast<float4 *>(dst + 32 * c);
+#pragma unroll
+                        for (int e = 0; e < 8; ++e)
+                            d4[e] = make_float4(fmaf(f, __uint_as_float(v1[4 * e]), __uint_as_float(v2[4 * e])),
+                                                fmaf(f, __uint_as_float(v1[4 * e + 1]), __uint_as_float(v2[4 * e + 1])),
+                                                fmaf(f, __uint_as_float(v1[4 * e + 2]), __uint_as_float(v2[4 * e + 2])),
+                                                fmaf(f, __uint_as_float(v1[4 * e + 3]), __uint_as_float(v2[4 * e + 3])));
+                    }
+                }
+            }
+            tc_fence_before_sync();
+            dt_bar_sync(half);   // operands and accumulators are free for the next tile
+        }
+    }
+
+    __syncthreads();
+    if (abort_flag && tid == 0) atomicOr(a.err, TC_ERR_DECODE_TIMEOUT);
+    if (warp == 0) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base_s, DT_TMEM_COLS);
+    }
+}
+
+float best_table_scale(const Codebook &cb, uint16_t (&table)[16]);
+
+bool decode_tc_supported(const eosq_cache_t &cache, int bits, const void *out_blocks) {
+    return bits == 2 && (reinterpret_cast<uintptr_t>(cache.codes) & 15u) == 0 && (reinterpret_cast<uintptr_t>(out_blocks) & 15u) == 0;
+}
+
+bool launch_decode_tc(const eosq_cache_t &cache, int64_t nb, int n, const Rotation &rot, const Codebook &cb, void *out_blocks,
+                      int out_dtype, int *err, int sm_count, cudaStream_t s) {
+    static bool configured = false;
+    if (!configured) {
+        if (cudaFuncSetAttribute(decode_tc_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(DT_SMEM)) != cudaSuccess ||
+            cudaFuncSetAttribute(decode_tc_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(DT_SMEM)) != cudaSuccess)
+            return false;
+        configured = true;
+    }
+    // the centroid table depends only on the codebook: search its scale once
+    static uint16_t table[16];
+    static float kappa = 0.0f;
+    static bool have_table = false;
+    if (!have_table) {
+        kappa = best_table_scale(cb, table);
+        have_table = true;
+    }
+    DecodeArgs a;
+    a.cache = cache;
+    a.nb = static_cast<int>(nb);
+    a.n = n;
+    a.inv_scale = 1.0f / (kappa * DT_PSCALE);
+    a.lo_tab = 0u;
+    a.hi_tab = 0u;
+    for (int k = 0; k < 4; ++k) {
+        a.lo_tab |= static_cast<uint32_t>(table[k] & 0xFFu) << (8 * k);
+        a.hi_tab |= static_cast<uint32_t>(table[k] >> 8) << (8 * k);
+    }
+    a.pi_t = rot.pi_t;
+    a.out = out_blocks;
+    a.err = err;
+    const int grid = static_cast<int>(std::min<int64_t>((nb + 1) / 2, sm_count));
+    if (out_dtype == EOSQ_F32)
+        decode_tc_kernel<float><<<grid, DT_THREADS, DT_SMEM, s>>>(a);
+    else
+        decode_tc_kernel<__half><<<grid, DT_THREADS, DT_SMEM, s>>>(a);
+    return true;
+}
+
+}  // namespace eosq

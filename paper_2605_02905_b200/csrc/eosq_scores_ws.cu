@@ -17,6 +17,7 @@
 
 #include "eosq_common.cuh"
 #include "eosq_sm100.cuh"
+#include "eosq_expand.cuh"
 
 namespace eosq {
 
@@ -63,30 +64,6 @@ __device__ __forceinline__ void ws_bulk_load(void *smem_dst, const void *gsrc, u
                  :
                  : "r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(gsrc)), "r"(bytes), "r"(smem_u32(bar))
                  : "memory");
-}
-
-__device__ __forceinline__ uint32_t ws_prmt(uint32_t a, uint32_t b, uint32_t sel) {
-    uint32_t d;
-    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
-    return d;
-}
-
-// Sixteen 2-bit codes (one word) -> eight words of fp16 pairs through the four-entry byte tables.
-__device__ __forceinline__ void ws_expand16(uint32_t w, uint32_t lo_tab, uint32_t hi_tab, uint32_t *out) {
-#pragma unroll
-    for (int part = 0; part < 2; ++part) {
-        uint32_t t = (w >> (16 * part)) & 0xFFFFu;
-        t = (t | (t << 8)) & 0x00FF00FFu;
-        t = (t | (t << 4)) & 0x0F0F0F0Fu;
-        t = (t | (t << 2)) & 0x33333333u;   // one nibble per code
-#pragma unroll
-        for (int quad = 0; quad < 2; ++quad) {
-            const uint32_t sel = t >> (16 * quad);
-            const uint32_t lows = ws_prmt(lo_tab, 0u, sel), highs = ws_prmt(hi_tab, 0u, sel);
-            out[4 * part + 2 * quad] = ws_prmt(lows, highs, 0x5140u);
-            out[4 * part + 2 * quad + 1] = ws_prmt(lows, highs, 0x7362u);
-        }
-    }
 }
 
 // Byte offset of element (row, k) of a K-major, 128-byte-swizzled operand with 16 rows per 64-wide K box.
@@ -426,10 +403,10 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
                     uint32_t av[32];
                     const uint32_t w0[4] = {c0.x, c0.y, c0.z, c0.w}, w1[4] = {c1.x, c1.y, c1.z, c1.w};
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) ws_expand16(w0[q], a.lo_tab, a.hi_tab, &av[8 * q]);
+                    for (int q = 0; q < 4; ++q) expand16_2bit(w0[q], a.lo_tab, a.hi_tab, &av[8 * q]);
                     tmem_st32(tb, av);
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) ws_expand16(w1[q], a.lo_tab, a.hi_tab, &av[8 * q]);
+                    for (int q = 0; q < 4; ++q) expand16_2bit(w1[q], a.lo_tab, a.hi_tab, &av[8 * q]);
                     tmem_st32(tb + 32, av);
                 }
                 tmem_st8(tb + WS_COL_P, pw);

@@ -128,6 +128,19 @@ def test_ragged_and_extreme_block_lengths(ctx, n):
     parity.compare_scores(cache, q, s, 2, 2, 2, 3, SEED, 1.0 / math.sqrt(128), pairs=[(0, 0), (1, 1)])
 
 
+@pytest.mark.parametrize("n", [136, 1000])
+def test_two_bit_decode_with_a_ragged_last_tile(ctx, n):
+    """The tensor-core decode (2-bit codes) on blocks whose length is not a multiple of its 128-token tile,
+    an odd number of blocks (the two halves of its CTA get different counts), both output types."""
+    w = synth.kv_cache_blocks("ragged2", layers=1, kv_heads=1, tokens=n, n=n, rank_hi=6, seed=70 + n)
+    blocks = torch.cat([w.blocks, w.blocks[:1] * 0.5], dim=0)   # 3 blocks
+    dev, cache = _encode(ctx, blocks, 2)
+    for out_dtype in (torch.float16, torch.float32):
+        dec = eosq.eosq_decode(ctx, cache, SEED, out_dtype=out_dtype)
+        parity.compare_decode(cache, dec, 2, SEED, tol=1e-4 if out_dtype == torch.float32 else 1e-3)
+    assert eosq.eosq_check_status(ctx, cache) == 0
+
+
 def test_many_blocks_cross_the_chunk_boundary_and_are_deterministic(ctx):
     """More blocks than one internal chunk: every block must equal its stand-alone encoding."""
     w = synth.kv_cache_blocks("chunks", layers=2, kv_heads=3, tokens=128 * 51, n=128, rank_hi=4, seed=50)
