@@ -13,6 +13,7 @@
 // turns 64 columns of one token's accumulators into rho D1 / (kappa 2^12) + D2 and stores them.
 #include <algorithm>
 #include <cstdint>
+#include <cstring>
 
 #include "eosq_common.cuh"
 #include "eosq_expand.cuh"
@@ -55,15 +56,21 @@ struct DecodeArgs {
 };
 
 // What a thread fetches from global memory for one tile: 64 codes of its token, the token's norm,
-// and (threads of the first column half only) the token's factor entries, packed.
+// and (threads of the first column half only) the token's factor entries.  The values stay as
+// loaded until the tile is built: a use right after the load would stall the warp for the whole
+// memory latency instead of letting it run behind the MMAs.
 struct DtTileRegs {
     uint4 codes;
-    uint4 p0, p1;
-    float rho;
+    unsigned short p[RMAX];
+    unsigned short rho;
 };
 
+bool make_block_tensor_map(const void *blocks, int64_t nb, int n, CUtensorMap *out);
+
+// `omap` (fp16 output only): the output as [nb][n][128] fp16 with boxes of 128 tokens x 64 coordinates,
+// 128-byte swizzled - the layout of the A tile, which doubles as the staging buffer of the stores.
 template <typename Tout>
-__global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeArgs a) {
+__global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeArgs a, const __grid_constant__ CUtensorMap omap) {
     extern __shared__ uint8_t dt_smem_raw[];
     __shared__ __align__(8) uint64_t mma_done[2];
     __shared__ uint32_t tmem_base_s;
@@ -121,28 +128,20 @@ __global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeAr
         const bool valid = tok < n;
         const size_t t = static_cast<size_t>(blk) * n + tok;
         g.codes = valid ? __ldg(reinterpret_cast<const uint4 *>(a.cache.codes + t * 32 + 16 * box)) : make_uint4(0u, 0u, 0u, 0u);
-        g.rho = valid ? __half2float(__ushort_as_half(a.cache.norms[t])) : 0.0f;
-        uint32_t pw[8];
+        g.rho = valid ? a.cache.norms[t] : static_cast<unsigned short>(0);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) pw[i] = 0u;
-        if (box == 0 && valid) {
-#pragma unroll
-            for (int i = 0; i < RMAX; ++i) {
-                if (i < rank) {
-                    const uint32_t v = Pg[(static_cast<size_t>(blk) * RMAX + i) * n + tok];
-                    pw[i >> 1] |= v << (16 * (i & 1));
-                }
-            }
-        }
-        g.p0 = make_uint4(pw[0], pw[1], pw[2], pw[3]);
-        g.p1 = make_uint4(pw[4], pw[5], pw[6], pw[7]);
+        for (int i = 0; i < RMAX; ++i)
+            g.p[i] = (box == 0 && valid && i < rank) ? Pg[(static_cast<size_t>(blk) * RMAX + i) * n + tok] : static_cast<unsigned short>(0);
         return g;
     };
 
     uint32_t phase = 0;
     bool alive = true;
-    for (long long blk = 2ll * blockIdx.x + half; blk < a.nb && alive; blk += 2ll * gridDim.x) {
-        const int rank = max(0, min(a.cache.rank[blk], RMAX));
+    const long long blk0 = 2ll * blockIdx.x + half, bstep = 2ll * gridDim.x;
+    int rank_next = (blk0 < a.nb) ? a.cache.rank[blk0] : 0;
+    for (long long blk = blk0; blk < a.nb && alive; blk += bstep) {
+        const int rank = max(0, min(rank_next, RMAX));
+        if (blk + bstep < a.nb) rank_next = a.cache.rank[blk + bstep];   // known long before the next block starts
         {   // B operand of D2: row j, K = i: zeta_i[j] (zero beyond the rank); this thread: row r, entries 8 box .. 8 box + 7
             uint32_t vw[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
@@ -164,11 +163,14 @@ __global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeAr
                     *reinterpret_cast<uint4 *>(hbase + DT_H_A + dt_offset(r, 8 * box + 2 * q + 1)) = make_uint4(o[4], o[5], o[6], o[7]);
                 }
                 if (box == 0) {   // A operand of D2: the token's factor entries
-                    *reinterpret_cast<uint4 *>(hbase + DT_H_P + dt_offset(r, 0)) = g.p0;
-                    *reinterpret_cast<uint4 *>(hbase + DT_H_P + dt_offset(r, 1)) = g.p1;
+                    uint32_t pw[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) pw[i] = static_cast<uint32_t>(g.p[2 * i]) | (static_cast<uint32_t>(g.p[2 * i + 1]) << 16);
+                    *reinterpret_cast<uint4 *>(hbase + DT_H_P + dt_offset(r, 0)) = make_uint4(pw[0], pw[1], pw[2], pw[3]);
+                    *reinterpret_cast<uint4 *>(hbase + DT_H_P + dt_offset(r, 1)) = make_uint4(pw[4], pw[5], pw[6], pw[7]);
                 }
             }
-            const float f = g.rho * a.inv_scale;
+            const float f = __half2float(__ushort_as_half(g.rho)) * a.inv_scale;
             fence_proxy_async_smem();   // the operands were written by ordinary stores and are read by the tensor core
             dt_bar_sync(half);
             if (ht == 0) {
@@ -200,7 +202,7 @@ __global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeAr
                 tmem_ld32(d1 + lane_off + 64u * box + 32u * c, v1);
                 tmem_ld32(d2 + lane_off + 64u * box + 32u * c, v2);
                 tmem_ld_wait();
-                if (tok < n) {
+                if (tok < n || sizeof(Tout) == 2) {   // rows past the end are clipped by the tensor store
                     if (sizeof(Tout) == 2) {
                         uint32_t pk[16];
 #pragma unroll
@@ -210,9 +212,12 @@ __global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeAr
                             pk[e] = static_cast<uint32_t>(__half_as_ushort(__float2half_rn(x0))) |
                                     (static_cast<uint32_t>(__half_as_ushort(__float2half_rn(x1))) << 16);
                         }
-                        uint4 *d4 = reinterpret_cast<uint4 *>(dst + 32 * c);
+                        // into the A tile (its MMAs are over), in the swizzled layout a tensor store turns back into rows:
+                        // a thread's own 16-byte stores to global memory would touch 32 sectors per warp instruction
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) d4[e] = make_uint4(pk[4 * e], pk[4 * e + 1], pk[4 * e + 2], pk[4 * e + 3]);
+                        for (int e = 0; e < 4; ++e)
+                            *reinterpret_cast<uint4 *>(hbase + DT_H_A + dt_offset(r, 8 * box + 4 * c + e)) =
+                                make_uint4(pk[4 * e], pk[4 * e + 1], pk[4 * e + 2], pk[4 * e + 3]);
                     } else {
                         float4 *d4 = reinterpret_cast<float4 *>(dst + 32 * c);
 #pragma unroll
@@ -224,11 +229,24 @@ __global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeAr
                     }
                 }
             }
-            tc_fence_before_sync();
+            if (sizeof(Tout) == 2) {
+                fence_proxy_async_smem();   // the staged tile was written by ordinary stores and is read by the copy engine
+                tc_fence_before_sync();
+                dt_bar_sync(half);
+                if (ht == 0) {
+                    tma_store_3d(&omap, hbase + DT_H_A, 0, tile * 128, static_cast<int>(blk));
+                    tma_store_3d(&omap, hbase + DT_H_A + DT_BOX, 64, tile * 128, static_cast<int>(blk));
+                    bulk_commit_group();
+                    bulk_wait_read_all();   // the tile has left shared memory (the global writes may still be in flight)
+                }
+            } else {
+                tc_fence_before_sync();
+            }
             dt_bar_sync(half);   // operands and accumulators are free for the next tile
         }
     }
 
+    if (sizeof(Tout) == 2 && ht == 0) bulk_wait_all();
     __syncthreads();
     if (abort_flag && tid == 0) atomicOr(a.err, TC_ERR_DECODE_TIMEOUT);
     if (warp == 0) {
@@ -275,10 +293,14 @@ bool launch_decode_tc(const eosq_cache_t &cache, int64_t nb, int n, const Rotati
     a.out = out_blocks;
     a.err = err;
     const int grid = static_cast<int>(std::min<int64_t>((nb + 1) / 2, sm_count));
-    if (out_dtype == EOSQ_F32)
-        decode_tc_kernel<float><<<grid, DT_THREADS, DT_SMEM, s>>>(a);
-    else
-        decode_tc_kernel<__half><<<grid, DT_THREADS, DT_SMEM, s>>>(a);
+    CUtensorMap omap;
+    std::memset(&omap, 0, sizeof(omap));
+    if (out_dtype == EOSQ_F32) {
+        decode_tc_kernel<float><<<grid, DT_THREADS, DT_SMEM, s>>>(a, omap);
+    } else {
+        if (!make_block_tensor_map(out_blocks, nb, n, &omap)) return false;
+        decode_tc_kernel<__half><<<grid, DT_THREADS, DT_SMEM, s>>>(a, omap);
+    }
     return true;
 }
 
