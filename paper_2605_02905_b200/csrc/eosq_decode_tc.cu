@@ -61,8 +61,8 @@ struct DecodeArgs {
 // memory latency instead of letting it run behind the MMAs.
 struct DtTileRegs {
     uint4 codes;
-    unsigned short p[RMAX];
-    unsigned short rho;
+    uint32_t p[RMAX];
+    uint32_t rho;
 };
 
 bool make_block_tensor_map(const void *blocks, int64_t nb, int n, CUtensorMap *out);
@@ -122,21 +122,24 @@ __global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeAr
     const uint16_t *Pg = a.cache.P;
     Tout *outp = static_cast<Tout *>(a.out);
 
+    // Loads only (no select on a loaded value): a token past the end reads the block's last token and
+    // is zeroed when the tile is built; factor rows beyond the rank are skipped by a uniform branch.
     auto fetch = [&](long long blk, int tile, int rank) {
         DtTileRegs g;
-        const int tok = tile * 128 + r;
-        const bool valid = tok < n;
+        const int tok = min(tile * 128 + r, n - 1);
         const size_t t = static_cast<size_t>(blk) * n + tok;
-        g.codes = valid ? __ldg(reinterpret_cast<const uint4 *>(a.cache.codes + t * 32 + 16 * box)) : make_uint4(0u, 0u, 0u, 0u);
-        g.rho = valid ? a.cache.norms[t] : static_cast<unsigned short>(0);
+        g.codes = __ldg(reinterpret_cast<const uint4 *>(a.cache.codes + t * 32 + 16 * box));
+        g.rho = a.cache.norms[t];
 #pragma unroll
-        for (int i = 0; i < RMAX; ++i)
-            g.p[i] = (box == 0 && valid && i < rank) ? Pg[(static_cast<size_t>(blk) * RMAX + i) * n + tok] : static_cast<unsigned short>(0);
+        for (int i = 0; i < RMAX; ++i) {
+            g.p[i] = 0u;
+            if (i < rank) g.p[i] = Pg[(static_cast<size_t>(blk) * RMAX + i) * n + tok];
+        }
         return g;
     };
 
     uint32_t phase = 0;
-    bool alive = true;
+    bool alive = true, store_pending = false;
     const long long blk0 = 2ll * blockIdx.x + half, bstep = 2ll * gridDim.x;
     int rank_next = (blk0 < a.nb) ? a.cache.rank[blk0] : 0;
     for (long long blk = blk0; blk < a.nb && alive; blk += bstep) {
@@ -153,24 +156,33 @@ __global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeAr
         }
         DtTileRegs g = fetch(blk, 0, rank);
         for (int tile = 0; tile < tiles; ++tile) {
+            const bool valid = tile * 128 + r < n;
             {   // A operand of D1: this token's 64 coordinates of column half `box`, as fp16 centroids
                 const uint32_t w[4] = {g.codes.x, g.codes.y, g.codes.z, g.codes.w};
+                uint32_t o[4][8];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) expand16_2bit(w[q], a.lo_tab, a.hi_tab, o[q]);
+                // the tile still holds the previous tile's output until the copy engine has read it: the
+                // expansion above ran in the shadow of that read
+                if (store_pending) {
+                    if (ht == 0) bulk_wait_read_all();
+                    dt_bar_sync(half);
+                    store_pending = false;
+                }
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
-                    uint32_t o[8];
-                    expand16_2bit(w[q], a.lo_tab, a.hi_tab, o);
-                    *reinterpret_cast<uint4 *>(hbase + DT_H_A + dt_offset(r, 8 * box + 2 * q)) = make_uint4(o[0], o[1], o[2], o[3]);
-                    *reinterpret_cast<uint4 *>(hbase + DT_H_A + dt_offset(r, 8 * box + 2 * q + 1)) = make_uint4(o[4], o[5], o[6], o[7]);
+                    *reinterpret_cast<uint4 *>(hbase + DT_H_A + dt_offset(r, 8 * box + 2 * q)) = make_uint4(o[q][0], o[q][1], o[q][2], o[q][3]);
+                    *reinterpret_cast<uint4 *>(hbase + DT_H_A + dt_offset(r, 8 * box + 2 * q + 1)) = make_uint4(o[q][4], o[q][5], o[q][6], o[q][7]);
                 }
                 if (box == 0) {   // A operand of D2: the token's factor entries
                     uint32_t pw[8];
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) pw[i] = static_cast<uint32_t>(g.p[2 * i]) | (static_cast<uint32_t>(g.p[2 * i + 1]) << 16);
+                    for (int i = 0; i < 8; ++i) pw[i] = valid ? (g.p[2 * i] | (g.p[2 * i + 1] << 16)) : 0u;
                     *reinterpret_cast<uint4 *>(hbase + DT_H_P + dt_offset(r, 0)) = make_uint4(pw[0], pw[1], pw[2], pw[3]);
                     *reinterpret_cast<uint4 *>(hbase + DT_H_P + dt_offset(r, 1)) = make_uint4(pw[4], pw[5], pw[6], pw[7]);
                 }
             }
-            const float f = __half2float(__ushort_as_half(g.rho)) * a.inv_scale;
+            const float f = valid ? __half2float(__ushort_as_half(static_cast<unsigned short>(g.rho))) * a.inv_scale : 0.0f;
             fence_proxy_async_smem();   // the operands were written by ordinary stores and are read by the tensor core
             dt_bar_sync(half);
             if (ht == 0) {
@@ -237,12 +249,12 @@ __global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeAr
                     tma_store_3d(&omap, hbase + DT_H_A, 0, tile * 128, static_cast<int>(blk));
                     tma_store_3d(&omap, hbase + DT_H_A + DT_BOX, 64, tile * 128, static_cast<int>(blk));
                     bulk_commit_group();
-                    bulk_wait_read_all();   // the tile has left shared memory (the global writes may still be in flight)
                 }
+                store_pending = true;   // waited for before the tile is overwritten
             } else {
                 tc_fence_before_sync();
+                dt_bar_sync(half);   // operands and accumulators are free for the next tile
             }
-            dt_bar_sync(half);   // operands and accumulators are free for the next tile
         }
     }
 
