@@ -359,6 +359,7 @@ def run_library(args):
 
 
 def main():
+    global BITS, WORKLOAD
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5)
@@ -368,8 +369,12 @@ def main():
     ap.add_argument("--e2e-blocks", type=int, default=None, help="blocks per end-to-end host-buffer call (default: the whole cache)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-decode", action="store_true")
+    ap.add_argument("--bits", type=int, default=BITS, choices=[1, 2, 3, 4],
+                    help="code width b (the headline configuration is b = 2; b = 3 is its second variant)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    BITS = args.bits
+    WORKLOAD = f"llama31_8b_T32768_n1024_d128_b{BITS}"
     if args.impl == "reference":
         run_reference(args)
     else:

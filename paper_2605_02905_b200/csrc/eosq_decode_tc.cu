@@ -1,4 +1,4 @@
-// Tensor-core decode for 2-bit codes (Algorithm 1 DeQuant + the stored low-rank part):
+// Tensor-core decode for 2- and 3-bit codes (Algorithm 1 DeQuant + the stored low-rank part):
 //   x_t = rho_t (z_t Pi) + sum_i P[t][i] zeta_i,     z_t = centroids of the codes of token t.
 //
 // One persistent CTA of 512 threads per SM holds the rotation once, as the B operand of
@@ -49,7 +49,7 @@ struct DecodeArgs {
     eosq_cache_t cache;
     int nb, n;
     float inv_scale;            // 1 / (kappa 2^12)
-    uint32_t lo_tab, hi_tab;    // bytes of the four fp16 centroids times kappa
+    uint32_t lo_tab[2], hi_tab[2];   // low / high bytes of the fp16 centroids times kappa (level k in byte k)
     const float *pi_t;          // pi_t[j][c] = Pi[c][j]
     void *out;
     int *err;
@@ -59,8 +59,9 @@ struct DecodeArgs {
 // and (threads of the first column half only) the token's factor entries.  The values stay as
 // loaded until the tile is built: a use right after the load would stall the warp for the whole
 // memory latency instead of letting it run behind the MMAs.
+template <int BITS>
 struct DtTileRegs {
-    uint4 codes;
+    uint32_t cw[2 * BITS];   // 64 codes
     uint32_t p[RMAX];
     uint32_t rho;
 };
@@ -69,8 +70,9 @@ bool make_block_tensor_map(const void *blocks, int64_t nb, int n, CUtensorMap *o
 
 // `omap` (fp16 output only): the output as [nb][n][128] fp16 with boxes of 128 tokens x 64 coordinates,
 // 128-byte swizzled - the layout of the A tile, which doubles as the staging buffer of the stores.
-template <typename Tout>
+template <typename Tout, int BITS>
 __global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeArgs a, const __grid_constant__ CUtensorMap omap) {
+    static_assert(BITS == 2 || BITS == 3, "byte-permute expansion covers up to eight levels");
     extern __shared__ uint8_t dt_smem_raw[];
     __shared__ __align__(8) uint64_t mma_done[2];
     __shared__ uint32_t tmem_base_s;
@@ -125,10 +127,18 @@ __global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeAr
     // Loads only (no select on a loaded value): a token past the end reads the block's last token and
     // is zeroed when the tile is built; factor rows beyond the rank are skipped by a uniform branch.
     auto fetch = [&](long long blk, int tile, int rank) {
-        DtTileRegs g;
+        DtTileRegs<BITS> g;
         const int tok = min(tile * 128 + r, n - 1);
         const size_t t = static_cast<size_t>(blk) * n + tok;
-        g.codes = __ldg(reinterpret_cast<const uint4 *>(a.cache.codes + t * 32 + 16 * box));
+        {   // the token's row is 16 BITS bytes; this thread's 64 codes are its half `box`
+            const uint2 *src = reinterpret_cast<const uint2 *>(a.cache.codes + t * (16 * BITS) + 8 * BITS * box);
+#pragma unroll
+            for (int w = 0; w < BITS; ++w) {
+                const uint2 v = __ldg(src + w);
+                g.cw[2 * w] = v.x;
+                g.cw[2 * w + 1] = v.y;
+            }
+        }
         g.rho = a.cache.norms[t];
 #pragma unroll
         for (int i = 0; i < RMAX; ++i) {
@@ -154,14 +164,13 @@ __global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeAr
             }
             *reinterpret_cast<uint4 *>(hbase + DT_H_V + dt_offset(r, box)) = make_uint4(vw[0], vw[1], vw[2], vw[3]);
         }
-        DtTileRegs g = fetch(blk, 0, rank);
+        DtTileRegs<BITS> g = fetch(blk, 0, rank);
         for (int tile = 0; tile < tiles; ++tile) {
             const bool valid = tile * 128 + r < n;
             {   // A operand of D1: this token's 64 coordinates of column half `box`, as fp16 centroids
-                const uint32_t w[4] = {g.codes.x, g.codes.y, g.codes.z, g.codes.w};
                 uint32_t o[4][8];
 #pragma unroll
-                for (int q = 0; q < 4; ++q) expand16_2bit(w[q], a.lo_tab, a.hi_tab, o[q]);
+                for (int q = 0; q < 4; ++q) expand16_codes<BITS>(g.cw, q, a.lo_tab, a.hi_tab, o[q]);
                 // the tile still holds the previous tile's output until the copy engine has read it: the
                 // expansion above ran in the shadow of that read
                 if (store_pending) {
@@ -270,36 +279,39 @@ __global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeAr
 float best_table_scale(const Codebook &cb, uint16_t (&table)[16]);
 
 bool decode_tc_supported(const eosq_cache_t &cache, int bits, const void *out_blocks) {
-    return bits == 2 && (reinterpret_cast<uintptr_t>(cache.codes) & 15u) == 0 && (reinterpret_cast<uintptr_t>(out_blocks) & 15u) == 0;
+    return (bits == 2 || bits == 3) && (reinterpret_cast<uintptr_t>(cache.codes) & 15u) == 0 &&
+           (reinterpret_cast<uintptr_t>(out_blocks) & 15u) == 0;
+}
+
+template <typename Tout, int BITS>
+static bool launch_decode_tc_as(const DecodeArgs &a, const CUtensorMap &omap, int grid, cudaStream_t s) {
+    static bool configured = false;
+    if (!configured) {
+        if (cudaFuncSetAttribute(decode_tc_kernel<Tout, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(DT_SMEM)) != cudaSuccess)
+            return false;
+        configured = true;
+    }
+    decode_tc_kernel<Tout, BITS><<<grid, DT_THREADS, DT_SMEM, s>>>(a, omap);
+    return true;
 }
 
 bool launch_decode_tc(const eosq_cache_t &cache, int64_t nb, int n, const Rotation &rot, const Codebook &cb, void *out_blocks,
                       int out_dtype, int *err, int sm_count, cudaStream_t s) {
-    static bool configured = false;
-    if (!configured) {
-        if (cudaFuncSetAttribute(decode_tc_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(DT_SMEM)) != cudaSuccess ||
-            cudaFuncSetAttribute(decode_tc_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(DT_SMEM)) != cudaSuccess)
-            return false;
-        configured = true;
-    }
-    // the centroid table depends only on the codebook: search its scale once
-    static uint16_t table[16];
-    static float kappa = 0.0f;
-    static bool have_table = false;
-    if (!have_table) {
-        kappa = best_table_scale(cb, table);
-        have_table = true;
-    }
+    // the centroid table depends only on the codebook: search its scale once per code width
+    static uint16_t table[5][16];
+    static float kappa[5] = {0.0f, 0.0f, 0.0f, 0.0f, 0.0f};
+    const int bits = cb.bits;
+    if (bits != 2 && bits != 3) return false;
+    if (kappa[bits] == 0.0f) kappa[bits] = best_table_scale(cb, table[bits]);
     DecodeArgs a;
     a.cache = cache;
     a.nb = static_cast<int>(nb);
     a.n = n;
-    a.inv_scale = 1.0f / (kappa * DT_PSCALE);
-    a.lo_tab = 0u;
-    a.hi_tab = 0u;
-    for (int k = 0; k < 4; ++k) {
-        a.lo_tab |= static_cast<uint32_t>(table[k] & 0xFFu) << (8 * k);
-        a.hi_tab |= static_cast<uint32_t>(table[k] >> 8) << (8 * k);
+    a.inv_scale = 1.0f / (kappa[bits] * DT_PSCALE);
+    a.lo_tab[0] = a.lo_tab[1] = a.hi_tab[0] = a.hi_tab[1] = 0u;
+    for (int k = 0; k < (1 << bits); ++k) {
+        a.lo_tab[k >> 2] |= static_cast<uint32_t>(table[bits][k] & 0xFFu) << (8 * (k & 3));
+        a.hi_tab[k >> 2] |= static_cast<uint32_t>(table[bits][k] >> 8) << (8 * (k & 3));
     }
     a.pi_t = rot.pi_t;
     a.out = out_blocks;
@@ -307,13 +319,10 @@ bool launch_decode_tc(const eosq_cache_t &cache, int64_t nb, int n, const Rotati
     const int grid = static_cast<int>(std::min<int64_t>((nb + 1) / 2, sm_count));
     CUtensorMap omap;
     std::memset(&omap, 0, sizeof(omap));
-    if (out_dtype == EOSQ_F32) {
-        decode_tc_kernel<float><<<grid, DT_THREADS, DT_SMEM, s>>>(a, omap);
-    } else {
-        if (!make_block_tensor_map(out_blocks, nb, n, &omap)) return false;
-        decode_tc_kernel<__half><<<grid, DT_THREADS, DT_SMEM, s>>>(a, omap);
-    }
-    return true;
+    if (out_dtype == EOSQ_F32)
+        return bits == 2 ? launch_decode_tc_as<float, 2>(a, omap, grid, s) : launch_decode_tc_as<float, 3>(a, omap, grid, s);
+    if (!make_block_tensor_map(out_blocks, nb, n, &omap)) return false;
+    return bits == 2 ? launch_decode_tc_as<__half, 2>(a, omap, grid, s) : launch_decode_tc_as<__half, 3>(a, omap, grid, s);
 }
 
 }  // namespace eosq
