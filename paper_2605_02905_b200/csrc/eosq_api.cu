@@ -318,7 +318,7 @@ extern "C" int eosq_scores(eosq_ctx *ctx, const eosq_cache_t *kcache, int64_t nu
     if ((rc = get_rotation(ctx, d, seed, &rot)) != EOSQ_OK) return rc;
     if ((rc = get_codebook(d, bits, &cb)) != EOSQ_OK) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    if (scores_tc_supported(bits, n) && (reinterpret_cast<uintptr_t>(kcache->codes) & 15u) == 0) {
+    if (scores_tc_supported(*kcache, bits, n) && (reinterpret_cast<uintptr_t>(kcache->codes) & 15u) == 0) {
         bool setup_ok = true;
         run_stage(ctx, ST_SCORES, s, [&] {
             setup_ok = launch_scores_tc(*kcache, num_kv_heads, blocks_per_head, head_stride_blocks, n, rot, cb,

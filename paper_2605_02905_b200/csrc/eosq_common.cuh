@@ -154,7 +154,7 @@ void launch_scores_plain(const eosq_cache_t &cache, int64_t heads, int64_t bph, 
                          float *scores, cudaStream_t s);
 
 // Tensor-core version of the logits (2-bit codes); returns false if nothing was enqueued.
-bool scores_tc_supported(int bits, int n);
+bool scores_tc_supported(const eosq_cache_t &cache, int bits, int n);
 bool launch_scores_tc(const eosq_cache_t &cache, int64_t heads, int64_t bph, int64_t head_stride, int n, const Rotation &rot,
                       const Codebook &cb, const __half *q, int G, float scale, float *scores, int *err, int sm_count,
                       cudaStream_t s);

@@ -327,11 +327,15 @@ float best_table_scale(const Codebook &cb, uint16_t (&table)[16]) {
 }
 
 bool scores_ws_supported(const eosq_cache_t &cache, int bits, int n);
-bool launch_scores_ws(const eosq_cache_t &cache, int64_t heads, int64_t bph, int64_t head_stride, int n, const Rotation &rot,
+bool launch_scores_ws(const eosq_cache_t &cache, int bits, int64_t heads, int64_t bph, int64_t head_stride, int n, const Rotation &rot,
                       const uint16_t (&table)[16], float kappa, const __half *q, int G, float scale, float *scores, int *err,
                       int sm_count, cudaStream_t s);
 
-bool scores_tc_supported(int bits, int n) { return bits == 2 && n >= 128; }
+// 2-bit codes always (the simpler kernel below takes what the warp-specialised one cannot); 3-bit codes
+// where the warp-specialised kernel applies.
+bool scores_tc_supported(const eosq_cache_t &cache, int bits, int n) {
+    return n >= 128 && (bits == 2 || (bits == 3 && scores_ws_supported(cache, bits, n)));
+}
 
 bool launch_scores_tc(const eosq_cache_t &cache, int64_t heads, int64_t bph, int64_t head_stride, int n, const Rotation &rot,
                       const Codebook &cb, const __half *q, int G, float scale, float *scores, int *err, int sm_count,
@@ -344,15 +348,15 @@ bool launch_scores_tc(const eosq_cache_t &cache, int64_t heads, int64_t bph, int
         configured = true;
     }
     // the table depends only on the codebook: search once per bit width
-    static uint16_t table[16];
-    static float kappa = 0.0f;
-    static int table_bits = 0;
-    if (table_bits != cb.bits) {
-        kappa = best_table_scale(cb, table);
-        table_bits = cb.bits;
-    }
+    static uint16_t tables[5][16];
+    static float kappas[5] = {0.0f, 0.0f, 0.0f, 0.0f, 0.0f};
+    if (cb.bits < 1 || cb.bits > 4) return false;
+    if (kappas[cb.bits] == 0.0f) kappas[cb.bits] = best_table_scale(cb, tables[cb.bits]);
+    const uint16_t (&table)[16] = tables[cb.bits];
+    const float kappa = kappas[cb.bits];
     if (scores_ws_supported(cache, cb.bits, n))
-        return launch_scores_ws(cache, heads, bph, head_stride, n, rot, table, kappa, q, G, scale, scores, err, sm_count, s);
+        return launch_scores_ws(cache, cb.bits, heads, bph, head_stride, n, rot, table, kappa, q, G, scale, scores, err, sm_count, s);
+    if (cb.bits != 2) return false;
     ScoresArgs a;
     a.cache = cache;
     a.bph = bph;

@@ -1,4 +1,4 @@
-// Warp-specialised attention-logit kernel for 2-bit codes (Remark 6.4): one persistent CTA of 16
+// Warp-specialised attention-logit kernel for 2- and 3-bit codes (Remark 6.4): one persistent CTA of 16
 // warps per SM in which loading, code expansion, the MMAs and the output run concurrently on
 // different tiles.
 //
@@ -31,28 +31,30 @@ constexpr int WS_STAGES = 5;               // shared-memory stages of WS_TPS til
 constexpr int WS_TPS = 4;                  // tiles per stage: few large copies keep the copy engine's queue short
 constexpr int WS_BUFS = 4;
 constexpr int WS_PMAX = 12;                // factor rows staged per tile (rank <= pilot k = 11)
-constexpr uint32_t WS_ST_CODES = 0, WS_ST_NORMS = 16384, WS_ST_P = 17408;   // 512 tokens: codes, norms, 2 boxes of 12 x 256 factors
+// a stage holds 512 tokens: codes (16 BITS bytes per token), norms, 2 boxes of 12 x 256 factors
+constexpr uint32_t WS_ST_CODES = 0;
 constexpr uint32_t WS_ST_PBOX = WS_PMAX * 512;
-constexpr uint32_t WS_STAGE_BYTES = WS_ST_P + 2 * WS_ST_PBOX;              // 29696
+template <int BITS> struct WsLayout {
+    static constexpr uint32_t ROW = 16 * BITS;                              // code bytes per token
+    static constexpr uint32_t ST_NORMS = 512 * ROW, ST_P = ST_NORMS + 1024;
+    static constexpr uint32_t STAGE_BYTES = ST_P + 2 * WS_ST_PBOX;         // 29696 (2 bits), 37888 (3 bits)
+    static constexpr uint32_t OFF_B1 = WS_STAGES * STAGE_BYTES;            // 2 x 4096: W, hi rows 0-7, lo rows 8-15
+    static constexpr uint32_t OFF_B2 = OFF_B1 + 2 * 4096;                  // 2 x 2048: Aq
+    static constexpr uint32_t OFF_V = OFF_B2 + 2 * 2048;                   // 2 x 4096: right vectors (fp16)
+    static constexpr uint32_t OFF_Q = OFF_V + 2 * 4096;                    // 2 x (8 x 128) fp32 queries, by head parity
+    static constexpr uint32_t SMEM_BYTES = OFF_Q + 2 * WS_NQ * D * 4 + 1024;
+};
 constexpr uint32_t WS_TMEM_COLS = 512;
 constexpr uint32_t WS_BUF_COLS = 112;      // per buffer: A 0-63, P 64-71, rho 72, D1 80-95, D2 96-111
 constexpr uint32_t WS_COL_P = 64, WS_COL_RHO = 72, WS_COL_D1 = 80, WS_COL_D2 = 96;
 constexpr float WS_QSCALE = 256.0f;
-
-// shared-memory map (offsets from a 1024-byte aligned base)
-constexpr uint32_t WS_OFF_STAGES = 0;
-constexpr uint32_t WS_OFF_B1 = WS_STAGES * WS_STAGE_BYTES;          // 2 x 4096: W, hi rows 0-7, lo rows 8-15
-constexpr uint32_t WS_OFF_B2 = WS_OFF_B1 + 2 * 4096;                // 2 x 2048: Aq
-constexpr uint32_t WS_OFF_V = WS_OFF_B2 + 2 * 2048;                 // 2 x 4096: right vectors (fp16)
-constexpr uint32_t WS_OFF_Q = WS_OFF_V + 2 * 4096;                  // 2 x (8 x 128) fp32 queries, by head parity
-constexpr uint32_t WS_SMEM_BYTES = WS_OFF_Q + 2 * WS_NQ * D * 4 + 1024;
 
 struct WsArgs {
     eosq_cache_t cache;
     int bph, head_stride, heads;   // blocks per head, block stride between heads, heads
     int n, G, g0;
     float scale, inv_code;
-    uint32_t lo_tab, hi_tab;
+    uint32_t lo_tab[2], hi_tab[2];   // low / high bytes of the fp16 centroids times kappa (level k in byte k)
     const float *pi_t;
     const __half *q;
     float *scores;
@@ -86,9 +88,11 @@ struct WsBarriers {
 
 bool make_factor_tensor_map(const void *P, int64_t nb, int n, int rows, CUtensorMap *out);
 
+template <int BITS>
 __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a, const __grid_constant__ CUtensorMap pmap4,
                                                                   const __grid_constant__ CUtensorMap pmap8,
                                                                   const __grid_constant__ CUtensorMap pmap12) {
+    using L = WsLayout<BITS>;
     extern __shared__ uint8_t ws_smem_raw[];
     __shared__ __align__(8) WsBarriers bars;
     __shared__ uint32_t tmem_base_s;
@@ -159,7 +163,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
                     alive = mbar_wait(&bars.blk_empty[vb], ((bi >> 1) & 1u) ^ 1u, &abort_flag);
                     if (alive) {
                         mbar_arrive_expect_tx(&bars.blk_full[vb], 4096);
-                        ws_bulk_load(base + WS_OFF_V + vb * 4096, a.cache.V + gb * RMAX * D, 4096, &bars.blk_full[vb]);
+                        ws_bulk_load(base + L::OFF_V + vb * 4096, a.cache.V + gb * RMAX * D, 4096, &bars.blk_full[vb]);
                     }
                 }
                 alive = __shfl_sync(0xffffffffu, alive, 0);
@@ -173,21 +177,21 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
                         alive = mbar_wait(&bars.st_empty[stage], ((sseq / WS_STAGES) & 1u) ^ 1u, &abort_flag);
                         if (alive) {
                             st_rank[stage] = rank;
-                            mbar_arrive_expect_tx(&bars.st_full[stage], rows * 34u + boxes * static_cast<uint32_t>(r4) * 2048u);
+                            mbar_arrive_expect_tx(&bars.st_full[stage], rows * (L::ROW + 2u) + boxes * static_cast<uint32_t>(r4) * 2048u);
                         }
                     }
                     alive = __shfl_sync(0xffffffffu, alive, 0);
                     if (!alive) break;
-                    uint8_t *st = base + WS_OFF_STAGES + stage * WS_STAGE_BYTES;
+                    uint8_t *st = base + stage * L::STAGE_BYTES;
                     const size_t t0 = static_cast<size_t>(gb) * n + tok0;
                     if (lane < 2) {
                         if (r4 > 0 && static_cast<uint32_t>(lane) < boxes)
-                            tma_load_3d(st + WS_ST_P + lane * WS_ST_PBOX, r4 == 1 ? &pmap4 : (r4 == 2 ? &pmap8 : &pmap12), &bars.st_full[stage],
+                            tma_load_3d(st + L::ST_P + lane * WS_ST_PBOX, r4 == 1 ? &pmap4 : (r4 == 2 ? &pmap8 : &pmap12), &bars.st_full[stage],
                                         tok0 + 256 * lane, 0, static_cast<int>(gb));
                     } else if (lane == 30)
-                        ws_bulk_load(st + WS_ST_CODES, a.cache.codes + t0 * 32, rows * 32, &bars.st_full[stage]);
+                        ws_bulk_load(st + WS_ST_CODES, a.cache.codes + t0 * L::ROW, rows * L::ROW, &bars.st_full[stage]);
                     else if (lane == 31)
-                        ws_bulk_load(st + WS_ST_NORMS, a.cache.norms + t0, rows * 2, &bars.st_full[stage]);
+                        ws_bulk_load(st + L::ST_NORMS, a.cache.norms + t0, rows * 2, &bars.st_full[stage]);
                 }
                 head = nhead;
                 jb = njb;
@@ -208,7 +212,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
                 }
                 const int vb = bi & 1, hb = hidx & 1;
                 if (!mbar_wait(&bars.b2_full[vb], (bi >> 1) & 1u, &abort_flag)) break;
-                const uint32_t b1 = smem_u32(base + WS_OFF_B1 + hb * 4096), b2 = smem_u32(base + WS_OFF_B2 + vb * 2048);
+                const uint32_t b1 = smem_u32(base + L::OFF_B1 + hb * 4096), b2 = smem_u32(base + L::OFF_B2 + vb * 2048);
                 uint64_t bdesc[D / 16 + 1];
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) bdesc[ks] = umma_desc_sw128(b1 + (ks >> 2) * 2048 + (ks & 3) * 32, 16, 1024);
@@ -243,7 +247,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
     } else if (warp < 4) {
         // ---------------------------------------------------------------- operand builder (64 threads)
         const int bt = tid - 64;
-        float *qs_all = reinterpret_cast<float *>(base + WS_OFF_Q);
+        float *qs_all = reinterpret_cast<float *>(base + L::OFF_Q);
         // W = Pi q of head `hd`, the `hx`-th head of this CTA, into the operand buffer of its parity
         auto build_w = [&](int hd, int hx) -> bool {
             const int hb = hx & 1;
@@ -254,7 +258,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
                 qs[e] = (g < gcount) ? __half2float(a.q[(static_cast<long long>(hd) * a.G + a.g0 + g) * D + (e % D)]) : 0.0f;
             }
             asm volatile("bar.sync 2, 64;" ::: "memory");
-            uint8_t *b1 = base + WS_OFF_B1 + hb * 4096;
+            uint8_t *b1 = base + L::OFF_B1 + hb * 4096;
             for (int rep = 0; rep < 2; ++rep) {
                 const int c = bt + 64 * rep;
                 float w[WS_NQ];
@@ -295,8 +299,8 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
             if (!mbar_wait(&bars.blk_full[vb], (bi >> 1) & 1u, &abort_flag) ||
                 !mbar_wait(&bars.b2_empty[vb], ((bi >> 1) & 1u) ^ 1u, &abort_flag))
                 break;
-            const __half *vs = reinterpret_cast<const __half *>(base + WS_OFF_V + vb * 4096);
-            uint8_t *b2 = base + WS_OFF_B2 + vb * 2048;
+            const __half *vs = reinterpret_cast<const __half *>(base + L::OFF_V + vb * 4096);
+            uint8_t *b2 = base + L::OFF_B2 + vb * 2048;
             for (int e = bt; e < WS_NQ * RMAX; e += 64) {   // Aq[g][i] = q_g . zeta_i
                 const int g = e >> 4, i = e & 15;
                 float dot = 0.0f;
@@ -359,14 +363,21 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
                     alive = false;
                     break;
                 }
-                const uint8_t *st = base + WS_OFF_STAGES + stage * WS_STAGE_BYTES;
+                const uint8_t *st = base + stage * L::STAGE_BYTES;
                 const int rank = st_rank[stage];
                 const bool valid = tile * 128 + wt < n;
                 const int st_tok = (tile % WS_TPS) * 128 + wt;   // token within the stage
-                uint4 c0 = *reinterpret_cast<const uint4 *>(st + WS_ST_CODES + st_tok * 32);
-                uint4 c1 = *reinterpret_cast<const uint4 *>(st + WS_ST_CODES + st_tok * 32 + 16);
-                unsigned short rho_raw = *reinterpret_cast<const unsigned short *>(st + WS_ST_NORMS + st_tok * 2);
-                const uint8_t *pcol = st + WS_ST_P + (st_tok >> 8) * WS_ST_PBOX + (st_tok & 255) * 2;
+                uint32_t cw[4 * BITS];   // the token's 128 codes
+#pragma unroll
+                for (int w = 0; w < BITS; ++w) {
+                    const uint4 v = *reinterpret_cast<const uint4 *>(st + WS_ST_CODES + st_tok * L::ROW + 16 * w);
+                    cw[4 * w] = v.x;
+                    cw[4 * w + 1] = v.y;
+                    cw[4 * w + 2] = v.z;
+                    cw[4 * w + 3] = v.w;
+                }
+                unsigned short rho_raw = *reinterpret_cast<const unsigned short *>(st + L::ST_NORMS + st_tok * 2);
+                const uint8_t *pcol = st + L::ST_P + (st_tok >> 8) * WS_ST_PBOX + (st_tok & 255) * 2;
                 uint32_t pw[8];
 #pragma unroll
                 for (int i = 0; i < 8; ++i) pw[i] = 0u;
@@ -385,8 +396,8 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
                         for (int r = 0; r < arrivals; ++r) mbar_arrive(&bars.st_empty[stage]);
                 }
                 if (!valid) {   // rows past the end of the block were not copied: the stage holds stale bytes there
-                    c0 = make_uint4(0u, 0u, 0u, 0u);
-                    c1 = c0;
+#pragma unroll
+                    for (int w = 0; w < 4 * BITS; ++w) cw[w] = 0u;
                     rho_raw = 0;
 #pragma unroll
                     for (int i = 0; i < 8; ++i) pw[i] = 0u;
@@ -401,12 +412,11 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
                 const uint32_t tb = tmem0 + lane_base + buf * WS_BUF_COLS;
                 {
                     uint32_t av[32];
-                    const uint32_t w0[4] = {c0.x, c0.y, c0.z, c0.w}, w1[4] = {c1.x, c1.y, c1.z, c1.w};
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) expand16_2bit(w0[q], a.lo_tab, a.hi_tab, &av[8 * q]);
+                    for (int q = 0; q < 4; ++q) expand16_codes<BITS>(cw, q, a.lo_tab, a.hi_tab, &av[8 * q]);
                     tmem_st32(tb, av);
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) expand16_2bit(w1[q], a.lo_tab, a.hi_tab, &av[8 * q]);
+                    for (int q = 0; q < 4; ++q) expand16_codes<BITS>(cw + 2 * BITS, q, a.lo_tab, a.hi_tab, &av[8 * q]);
                     tmem_st32(tb + 32, av);
                 }
                 tmem_st8(tb + WS_COL_P, pw);
@@ -481,19 +491,29 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
 
 bool scores_ws_supported(const eosq_cache_t &cache, int bits, int n) {
     auto aligned = [](const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; };
-    return bits == 2 && n >= 128 && (n % 8) == 0 && aligned(cache.codes) && aligned(cache.norms) && aligned(cache.P) && aligned(cache.V);
+    return (bits == 2 || bits == 3) && n >= 128 && (n % 8) == 0 && aligned(cache.codes) && aligned(cache.norms) && aligned(cache.P) && aligned(cache.V);
 }
 
-bool launch_scores_ws(const eosq_cache_t &cache, int64_t heads, int64_t bph, int64_t head_stride, int n, const Rotation &rot,
-                      const uint16_t (&table)[16], float kappa, const __half *q, int G, float scale, float *scores, int *err,
-                      int sm_count, cudaStream_t s) {
+template <int BITS>
+static bool launch_scores_ws_as(WsArgs &a, int G, int grid, const CUtensorMap &m4, const CUtensorMap &m8, const CUtensorMap &m12, cudaStream_t s) {
     static bool configured = false;
     if (!configured) {
-        if (cudaFuncSetAttribute(scores_ws_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(WS_SMEM_BYTES)) != cudaSuccess)
+        if (cudaFuncSetAttribute(scores_ws_kernel<BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(WsLayout<BITS>::SMEM_BYTES)) != cudaSuccess)
             return false;
         configured = true;
     }
-    if (heads * bph > 0x7fffffff || head_stride > 0x7fffffff) return false;
+    for (int g0 = 0; g0 < G; g0 += WS_NQ) {
+        a.g0 = g0;
+        scores_ws_kernel<BITS><<<grid, WS_THREADS, WsLayout<BITS>::SMEM_BYTES, s>>>(a, m4, m8, m12);
+    }
+    return true;
+}
+
+bool launch_scores_ws(const eosq_cache_t &cache, int bits, int64_t heads, int64_t bph, int64_t head_stride, int n, const Rotation &rot,
+                      const uint16_t (&table)[16], float kappa, const __half *q, int G, float scale, float *scores, int *err,
+                      int sm_count, cudaStream_t s) {
+    if (heads * bph > 0x7fffffff || head_stride > 0x7fffffff || (bits != 2 && bits != 3)) return false;
     WsArgs a;
     a.cache = cache;
     a.bph = static_cast<int>(bph);
@@ -503,11 +523,10 @@ bool launch_scores_ws(const eosq_cache_t &cache, int64_t heads, int64_t bph, int
     a.G = G;
     a.scale = scale;
     a.inv_code = 1.0f / (kappa * WS_QSCALE);
-    a.lo_tab = 0u;
-    a.hi_tab = 0u;
-    for (int k = 0; k < 4; ++k) {
-        a.lo_tab |= static_cast<uint32_t>(table[k] & 0xFFu) << (8 * k);
-        a.hi_tab |= static_cast<uint32_t>(table[k] >> 8) << (8 * k);
+    a.lo_tab[0] = a.lo_tab[1] = a.hi_tab[0] = a.hi_tab[1] = 0u;
+    for (int k = 0; k < (1 << bits); ++k) {
+        a.lo_tab[k >> 2] |= static_cast<uint32_t>(table[k] & 0xFFu) << (8 * (k & 3));
+        a.hi_tab[k >> 2] |= static_cast<uint32_t>(table[k] >> 8) << (8 * (k & 3));
     }
     a.pi_t = rot.pi_t;
     a.q = q;
@@ -519,11 +538,7 @@ bool launch_scores_ws(const eosq_cache_t &cache, int64_t heads, int64_t bph, int
     if (!make_factor_tensor_map(cache.P, nb_total, n, 4, &m4) || !make_factor_tensor_map(cache.P, nb_total, n, 8, &m8) ||
         !make_factor_tensor_map(cache.P, nb_total, n, 12, &m12))
         return false;
-    for (int g0 = 0; g0 < G; g0 += WS_NQ) {
-        a.g0 = g0;
-        scores_ws_kernel<<<grid, WS_THREADS, WS_SMEM_BYTES, s>>>(a, m4, m8, m12);
-    }
-    return true;
+    return bits == 2 ? launch_scores_ws_as<2>(a, G, grid, m4, m8, m12, s) : launch_scores_ws_as<3>(a, G, grid, m4, m8, m12, s);
 }
 
 }  // namespace eosq
