@@ -340,7 +340,7 @@ extern "C" int eosq_scores(eosq_ctx *ctx, const eosq_cache_t *kcache, int64_t nu
 
 // ---- host-buffer path ----------------------------------------------------------------------
 namespace {
-constexpr int64_t HOST_CHUNK = 1184;
+constexpr int64_t HOST_CHUNK = 592;   // one encode chunk: a short pipeline fill (the first upload overlaps nothing)
 
 // Two slots (input chunk + its outputs) so that the upload of chunk i + 1 and the download of chunk
 // i - 1 run while chunk i is encoded, and one workspace (encodes run one after another).
