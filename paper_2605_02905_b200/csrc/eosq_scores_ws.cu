@@ -285,6 +285,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
         };
         int head = (it0 < it1) ? it0 / a.bph : 0, jb = it0 - head * a.bph, hidx = -1, prev_head = -1;
         bool first_of_head = false;
+        int rank_next = (it0 < it1) ? min(__ldg(a.cache.rank + static_cast<long long>(head) * a.head_stride + jb), WS_PMAX) : 0;
         for (int item = it0, bi = 0; item < it1; ++item, ++bi) {
             if (head != prev_head) {
                 hidx += 1;
@@ -295,39 +296,57 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
             const float *qs = qs_all + (hidx & 1) * WS_NQ * D;
             const long long gb = static_cast<long long>(head) * a.head_stride + jb;
             const int vb = bi & 1;
-            const int rank = min(__ldg(a.cache.rank + gb), WS_PMAX);
+            const int rank = rank_next;
+            {   // the next block's rank is asked for now: a load on the critical path of every block costs over 1 000 cycles
+                int nh = head, nj = jb + 1;
+                if (nj == a.bph) {
+                    nj = 0;
+                    nh += 1;
+                }
+                if (item + 1 < it1) rank_next = min(__ldg(a.cache.rank + static_cast<long long>(nh) * a.head_stride + nj), WS_PMAX);
+            }
             if (!mbar_wait(&bars.blk_full[vb], (bi >> 1) & 1u, &abort_flag) ||
                 !mbar_wait(&bars.b2_empty[vb], ((bi >> 1) & 1u) ^ 1u, &abort_flag))
                 break;
             const __half *vs = reinterpret_cast<const __half *>(base + L::OFF_V + vb * 4096);
             uint8_t *b2 = base + L::OFF_B2 + vb * 2048;
-            for (int e = bt; e < WS_NQ * RMAX; e += 64) {   // Aq[g][i] = q_g . zeta_i
+            // Aq[g][i] = q_g . zeta_i for g < gcount, i < rank, zero elsewhere.  Four lanes share a dot product
+            // (16-byte chunks of the row dealt round-robin, rotated by the dot's number so that the lanes of a warp
+            // hit different banks), sixteen dot products per round of the 64 threads.
+            for (int e = bt; e < WS_NQ * RMAX; e += 64) {
                 const int g = e >> 4, i = e & 15;
-                float dot = 0.0f;
-                if (i < rank && g < gcount) {
-                    const uint4 *vrow = reinterpret_cast<const uint4 *>(vs + i * D);
-                    const float4 *qrow = reinterpret_cast<const float4 *>(qs + g * D);
-                    float d0 = 0.0f, d1 = 0.0f;
-#pragma unroll 4
-                    for (int j = 0; j < D / 8; ++j) {
-                        const uint4 v = vrow[j];
-                        const float4 qa = qrow[2 * j], qb = qrow[2 * j + 1];
-                        const float2 v0 = __half22float2(*reinterpret_cast<const __half2 *>(&v.x));
-                        const float2 v1 = __half22float2(*reinterpret_cast<const __half2 *>(&v.y));
-                        const float2 v2 = __half22float2(*reinterpret_cast<const __half2 *>(&v.z));
-                        const float2 v3 = __half22float2(*reinterpret_cast<const __half2 *>(&v.w));
-                        d0 = fmaf(qa.x, v0.x, d0);
-                        d1 = fmaf(qa.y, v0.y, d1);
-                        d0 = fmaf(qa.z, v1.x, d0);
-                        d1 = fmaf(qa.w, v1.y, d1);
-                        d0 = fmaf(qb.x, v2.x, d0);
-                        d1 = fmaf(qb.y, v2.y, d1);
-                        d0 = fmaf(qb.z, v3.x, d0);
-                        d1 = fmaf(qb.w, v3.y, d1);
-                    }
-                    dot = d0 + d1;
+                if (!(i < rank && g < gcount)) ws_split_store(b2, g, i, 0.0f);
+            }
+            const int ndots = rank * gcount, part = bt & 3;
+            for (int d0i = 0; d0i < ndots; d0i += 16) {
+                const int dn = d0i + (bt >> 2);
+                const bool act = dn < ndots;
+                const int g = act ? dn / rank : 0, i = act ? dn - g * rank : 0;
+                const uint4 *vrow = reinterpret_cast<const uint4 *>(vs + i * D);
+                const float4 *qrow = reinterpret_cast<const float4 *>(qs + g * D);
+                float d0 = 0.0f, d1 = 0.0f;
+#pragma unroll
+                for (int it = 0; it < 4; ++it) {
+                    const int j = (4 * it + part + dn) & 15;
+                    const uint4 v = vrow[j];
+                    const float4 qa = qrow[2 * j], qb = qrow[2 * j + 1];
+                    const float2 v0 = __half22float2(*reinterpret_cast<const __half2 *>(&v.x));
+                    const float2 v1 = __half22float2(*reinterpret_cast<const __half2 *>(&v.y));
+                    const float2 v2 = __half22float2(*reinterpret_cast<const __half2 *>(&v.z));
+                    const float2 v3 = __half22float2(*reinterpret_cast<const __half2 *>(&v.w));
+                    d0 = fmaf(qa.x, v0.x, d0);
+                    d1 = fmaf(qa.y, v0.y, d1);
+                    d0 = fmaf(qa.z, v1.x, d0);
+                    d1 = fmaf(qa.w, v1.y, d1);
+                    d0 = fmaf(qb.x, v2.x, d0);
+                    d1 = fmaf(qb.y, v2.y, d1);
+                    d0 = fmaf(qb.z, v3.x, d0);
+                    d1 = fmaf(qb.w, v3.y, d1);
                 }
-                ws_split_store(b2, g, i, dot * WS_QSCALE);
+                float dot = d0 + d1;
+                dot += __shfl_xor_sync(0xffffffffu, dot, 1);
+                dot += __shfl_xor_sync(0xffffffffu, dot, 2);
+                if (act && part == 0) ws_split_store(b2, g, i, dot * WS_QSCALE);
             }
             fence_proxy_async_smem();
             asm volatile("bar.sync 2, 64;" ::: "memory");
