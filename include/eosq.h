@@ -176,6 +176,9 @@ int eosq_decode(eosq_ctx *ctx, const eosq_cache_t *cache, int64_t num_blocks, in
  * out [head][K|V][block]).
  *   q       dev [num_kv_heads][G][d] fp16
  *   scores  dev [num_kv_heads][G][blocks_per_head*n] fp32
+ * The tensor-core path keeps the rotated queries in a device buffer of 4 KB per KV head that the
+ * context owns: the first call (and a later call with more heads) allocates it, which synchronises
+ * the device; calls on one context must not overlap in time.
  */
 int eosq_scores(eosq_ctx *ctx, const eosq_cache_t *kcache, int64_t num_kv_heads,
                 int64_t blocks_per_head, int64_t head_stride_blocks, int n, int d, int bits,

@@ -197,6 +197,7 @@ extern "C" int eosq_destroy(eosq_ctx *ctx) {
         cudaEventDestroy(t.stop);
     }
     for (cudaEvent_t e : ctx->free_events) cudaEventDestroy(e);
+    cudaFree(ctx->scores_w);
     if (ctx->copy_in) cudaStreamDestroy(ctx->copy_in);
     if (ctx->copy_out) cudaStreamDestroy(ctx->copy_out);
     if (ctx->ev_start) cudaEventDestroy(ctx->ev_start);
@@ -322,7 +323,8 @@ extern "C" int eosq_scores(eosq_ctx *ctx, const eosq_cache_t *kcache, int64_t nu
         bool setup_ok = true;
         run_stage(ctx, ST_SCORES, s, [&] {
             setup_ok = launch_scores_tc(*kcache, num_kv_heads, blocks_per_head, head_stride_blocks, n, rot, cb,
-                                        static_cast<const __half *>(q), G, scale, scores, ctx->dev_err, ctx->sm_count, s);
+                                        static_cast<const __half *>(q), G, scale, scores, ctx->dev_err, ctx->sm_count, &ctx->scores_w,
+                                        &ctx->scores_w_bytes, s);
         });
         if (!setup_ok) {
             ctx->last_error = "tensor-core score kernel: launch set-up failed";

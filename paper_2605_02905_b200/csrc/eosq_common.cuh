@@ -99,6 +99,8 @@ struct eosq_ctx {
     uint32_t profile_mask = 0;   // bit i set: launches of stage i are bracketed by events
     std::vector<Timed> timed;
     std::vector<cudaEvent_t> free_events;
+    void *scores_w = nullptr;        // score path: per-head images of the operand W = Pi q (grown on demand)
+    size_t scores_w_bytes = 0;
     // host-buffer path: copy streams and hand-over events of its two arena slots (created on first use)
     cudaStream_t copy_in = nullptr, copy_out = nullptr;
     cudaEvent_t ev_start = nullptr, ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
@@ -157,7 +159,7 @@ void launch_scores_plain(const eosq_cache_t &cache, int64_t heads, int64_t bph, 
 bool scores_tc_supported(const eosq_cache_t &cache, int bits, int n);
 bool launch_scores_tc(const eosq_cache_t &cache, int64_t heads, int64_t bph, int64_t head_stride, int n, const Rotation &rot,
                       const Codebook &cb, const __half *q, int G, float scale, float *scores, int *err, int sm_count,
-                      cudaStream_t s);
+                      void **scratch, size_t *scratch_bytes, cudaStream_t s);
 
 // ---- small device helpers -------------------------------------------------------------------
 __device__ __forceinline__ double warp_sum(double v) {

@@ -55,7 +55,7 @@ struct WsArgs {
     int n, G, g0;
     float scale, inv_code;
     uint32_t lo_tab[2], hi_tab[2];   // low / high bytes of the fp16 centroids times kappa (level k in byte k)
-    const float *pi_t;
+    const uint8_t *wimg;   // per head: the 4096-byte image of the operand W = Pi q (made by scores_w_kernel)
     const __half *q;
     float *scores;
     int *err;
@@ -87,6 +87,30 @@ struct WsBarriers {
 };
 
 bool make_factor_tensor_map(const void *P, int64_t nb, int n, int rows, CUtensorMap *out);
+
+// W = Pi q for the (at most eight) query vectors g0.. of every head, times 2^8, split into a high and a low
+// fp16 plane and laid out as the score kernel's B operand (rows g and 8 + g of a K-major, 128-byte-swizzled
+// tile of 16 rows x 128): one 4096-byte image per head, which the score kernel fetches with one bulk copy.
+__global__ void __launch_bounds__(D) scores_w_kernel(const float *__restrict__ pi_t, const __half *__restrict__ q, int G, int g0,
+                                                     uint8_t *__restrict__ wimg) {
+    __shared__ float qs[WS_NQ][D];
+    const int c = threadIdx.x, hd = blockIdx.x;
+    const int gcount = min(WS_NQ, G - g0);
+    for (int g = 0; g < WS_NQ; ++g) qs[g][c] = (g < gcount) ? __half2float(q[(static_cast<long long>(hd) * G + g0 + g) * D + c]) : 0.0f;
+    __syncthreads();
+    float w[WS_NQ];
+#pragma unroll
+    for (int g = 0; g < WS_NQ; ++g) w[g] = 0.0f;
+#pragma unroll 4
+    for (int j = 0; j < D; ++j) {
+        const float pv = __ldg(pi_t + j * D + c);
+#pragma unroll
+        for (int g = 0; g < WS_NQ; ++g) w[g] = fmaf(pv, qs[g][j], w[g]);
+    }
+    uint8_t *img = wimg + static_cast<size_t>(hd) * 4096;
+#pragma unroll
+    for (int g = 0; g < WS_NQ; ++g) ws_split_store(img, g, c, w[g] * WS_QSCALE);
+}
 
 template <int BITS>
 __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a, const __grid_constant__ CUtensorMap pmap4,
@@ -248,39 +272,21 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
         // ---------------------------------------------------------------- operand builder (64 threads)
         const int bt = tid - 64;
         float *qs_all = reinterpret_cast<float *>(base + L::OFF_Q);
-        // W = Pi q of head `hd`, the `hx`-th head of this CTA, into the operand buffer of its parity
+        // Head `hd`, the `hx`-th head of this CTA: its queries into shared memory (for the Aq products) and the
+        // prepared image of W = Pi q, by one bulk copy, into the operand buffer of its parity.
         auto build_w = [&](int hd, int hx) -> bool {
             const int hb = hx & 1;
             float *qs = qs_all + hb * WS_NQ * D;
             if (!mbar_wait(&bars.b1_empty[hb], ((hx >> 1) & 1u) ^ 1u, &abort_flag)) return false;
+            if (bt == 0) {
+                mbar_arrive_expect_tx(&bars.b1_full[hb], 4096);
+                ws_bulk_load(base + L::OFF_B1 + hb * 4096, a.wimg + static_cast<size_t>(hd) * 4096, 4096, &bars.b1_full[hb]);
+            }
             for (int e = bt; e < WS_NQ * D; e += 64) {
                 const int g = e / D;
                 qs[e] = (g < gcount) ? __half2float(a.q[(static_cast<long long>(hd) * a.G + a.g0 + g) * D + (e % D)]) : 0.0f;
             }
             asm volatile("bar.sync 2, 64;" ::: "memory");
-            uint8_t *b1 = base + L::OFF_B1 + hb * 4096;
-            for (int rep = 0; rep < 2; ++rep) {
-                const int c = bt + 64 * rep;
-                float w[WS_NQ];
-#pragma unroll
-                for (int g = 0; g < WS_NQ; ++g) w[g] = 0.0f;
-#pragma unroll 1
-                for (int j0 = 0; j0 < D; j0 += 32) {
-                    float pv[32];
-#pragma unroll
-                    for (int jj = 0; jj < 32; ++jj) pv[jj] = __ldg(a.pi_t + (j0 + jj) * D + c);   // 32 loads in flight
-#pragma unroll
-                    for (int jj = 0; jj < 32; ++jj) {
-#pragma unroll
-                        for (int g = 0; g < WS_NQ; ++g) w[g] = fmaf(pv[jj], qs[g * D + j0 + jj], w[g]);
-                    }
-                }
-#pragma unroll
-                for (int g = 0; g < WS_NQ; ++g) ws_split_store(b1, g, c, w[g] * WS_QSCALE);
-            }
-            fence_proxy_async_smem();
-            asm volatile("bar.sync 2, 64;" ::: "memory");
-            if (bt == 0) mbar_arrive(&bars.b1_full[hb]);
             return true;
         };
         int head = (it0 < it1) ? it0 / a.bph : 0, jb = it0 - head * a.bph, hidx = -1, prev_head = -1;
@@ -514,7 +520,8 @@ bool scores_ws_supported(const eosq_cache_t &cache, int bits, int n) {
 }
 
 template <int BITS>
-static bool launch_scores_ws_as(WsArgs &a, int G, int grid, const CUtensorMap &m4, const CUtensorMap &m8, const CUtensorMap &m12, cudaStream_t s) {
+static bool launch_scores_ws_as(WsArgs &a, int G, int grid, const CUtensorMap &m4, const CUtensorMap &m8, const CUtensorMap &m12,
+                                const float *pi_t, uint8_t *wimg, cudaStream_t s) {
     static bool configured = false;
     if (!configured) {
         if (cudaFuncSetAttribute(scores_ws_kernel<BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -524,6 +531,7 @@ static bool launch_scores_ws_as(WsArgs &a, int G, int grid, const CUtensorMap &m
     }
     for (int g0 = 0; g0 < G; g0 += WS_NQ) {
         a.g0 = g0;
+        scores_w_kernel<<<a.heads, D, 0, s>>>(pi_t, a.q, G, g0, wimg);
         scores_ws_kernel<BITS><<<grid, WS_THREADS, WsLayout<BITS>::SMEM_BYTES, s>>>(a, m4, m8, m12);
     }
     return true;
@@ -531,7 +539,7 @@ static bool launch_scores_ws_as(WsArgs &a, int G, int grid, const CUtensorMap &m
 
 bool launch_scores_ws(const eosq_cache_t &cache, int bits, int64_t heads, int64_t bph, int64_t head_stride, int n, const Rotation &rot,
                       const uint16_t (&table)[16], float kappa, const __half *q, int G, float scale, float *scores, int *err,
-                      int sm_count, cudaStream_t s) {
+                      int sm_count, void **scratch, size_t *scratch_bytes, cudaStream_t s) {
     if (heads * bph > 0x7fffffff || head_stride > 0x7fffffff || (bits != 2 && bits != 3)) return false;
     WsArgs a;
     a.cache = cache;
@@ -547,7 +555,17 @@ bool launch_scores_ws(const eosq_cache_t &cache, int bits, int64_t heads, int64_
         a.lo_tab[k >> 2] |= static_cast<uint32_t>(table[k] & 0xFFu) << (8 * (k & 3));
         a.hi_tab[k >> 2] |= static_cast<uint32_t>(table[k] >> 8) << (8 * (k & 3));
     }
-    a.pi_t = rot.pi_t;
+    // one 4096-byte operand image per head, in a buffer the context keeps and grows (earlier work that
+    // still reads the old buffer is waited for by cudaFree)
+    const size_t need = static_cast<size_t>(heads) * 4096;
+    if (*scratch_bytes < need) {
+        cudaFree(*scratch);
+        *scratch = nullptr;
+        *scratch_bytes = 0;
+        if (cudaMalloc(scratch, need) != cudaSuccess) return false;
+        *scratch_bytes = need;
+    }
+    a.wimg = static_cast<const uint8_t *>(*scratch);
     a.q = q;
     a.scores = scores;
     a.err = err;
@@ -557,7 +575,9 @@ bool launch_scores_ws(const eosq_cache_t &cache, int bits, int64_t heads, int64_
     if (!make_factor_tensor_map(cache.P, nb_total, n, 4, &m4) || !make_factor_tensor_map(cache.P, nb_total, n, 8, &m8) ||
         !make_factor_tensor_map(cache.P, nb_total, n, 12, &m12))
         return false;
-    return bits == 2 ? launch_scores_ws_as<2>(a, G, grid, m4, m8, m12, s) : launch_scores_ws_as<3>(a, G, grid, m4, m8, m12, s);
+    uint8_t *wimg = static_cast<uint8_t *>(*scratch);
+    return bits == 2 ? launch_scores_ws_as<2>(a, G, grid, m4, m8, m12, rot.pi_t, wimg, s)
+                     : launch_scores_ws_as<3>(a, G, grid, m4, m8, m12, rot.pi_t, wimg, s);
 }
 
 }  // namespace eosq
