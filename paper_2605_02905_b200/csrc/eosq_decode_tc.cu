@@ -30,9 +30,15 @@ constexpr float DT_PSCALE = 4096.0f;                  // keeps the low plane of 
 constexpr uint32_t DT_BOX = 128 * 128;                // 128 rows x 64 fp16 of K
 constexpr uint32_t DT_OFF_PI_HI = 0, DT_OFF_PI_LO = 2 * DT_BOX;
 constexpr uint32_t DT_OFF_HALF = 4 * DT_BOX;          // per half: A tile (2 boxes), factor tile (1 box), right vectors (1 box)
-constexpr uint32_t DT_HALF_BYTES = 4 * DT_BOX;
 constexpr uint32_t DT_H_A = 0, DT_H_P = 2 * DT_BOX, DT_H_V = 3 * DT_BOX;
-constexpr size_t DT_SMEM = DT_OFF_HALF + 2 * DT_HALF_BYTES + 1024;   // 193 KB
+// ... and the raw data of the next tile, copied in while the current one is worked on: packed codes
+// (128 tokens x up to 48 bytes), norms, up to 12 factor rows of 128 fp16
+constexpr int DT_PMAX = 12;
+constexpr uint32_t DT_H_RAW = 4 * DT_BOX, DT_RAW_NORMS = 128 * 48, DT_RAW_P = DT_RAW_NORMS + 256;
+constexpr uint32_t DT_RAW_BYTES = 10240;
+static_assert(DT_RAW_P + DT_PMAX * 256 <= DT_RAW_BYTES && KPILOT < DT_PMAX, "the raw area holds one tile");
+constexpr uint32_t DT_HALF_BYTES = 4 * DT_BOX + DT_RAW_BYTES;
+constexpr size_t DT_SMEM = DT_OFF_HALF + 2 * DT_HALF_BYTES + 1024;   // 213 KB
 constexpr uint32_t DT_TMEM_COLS = 512;                // per half: D1 128 columns, D2 128 columns
 
 // Byte offset of the 16-byte chunk `jc` (8 fp16 of K) of row `row` in a K-major, 128-byte-swizzled
@@ -55,16 +61,12 @@ struct DecodeArgs {
     int *err;
 };
 
-// What a thread fetches from global memory for one tile: 64 codes of its token, the token's norm,
-// and (threads of the first column half only) the token's factor entries.  The values stay as
-// loaded until the tile is built: a use right after the load would stall the warp for the whole
-// memory latency instead of letting it run behind the MMAs.
-template <int BITS>
-struct DtTileRegs {
-    uint32_t cw[2 * BITS];   // 64 codes
-    uint32_t p[RMAX];
-    uint32_t rho;
-};
+__device__ __forceinline__ void dt_bulk_load(void *smem_dst, const void *gsrc, uint32_t bytes, uint64_t *bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :
+                 : "r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(gsrc)), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
 
 bool make_block_tensor_map(const void *blocks, int64_t nb, int n, CUtensorMap *out);
 
@@ -74,7 +76,7 @@ template <typename Tout, int BITS>
 __global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeArgs a, const __grid_constant__ CUtensorMap omap) {
     static_assert(BITS == 2 || BITS == 3, "byte-permute expansion covers up to eight levels");
     extern __shared__ uint8_t dt_smem_raw[];
-    __shared__ __align__(8) uint64_t mma_done[2];
+    __shared__ __align__(8) uint64_t mma_done[2], raw_full[2];
     __shared__ uint32_t tmem_base_s;
     __shared__ volatile int abort_flag;
 
@@ -87,6 +89,8 @@ __global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeAr
     if (tid == 0) {
         mbar_init(&mma_done[0], 1);
         mbar_init(&mma_done[1], 1);
+        mbar_init(&raw_full[0], 1);
+        mbar_init(&raw_full[1], 1);
         abort_flag = 0;
         fence_mbar_init();
     }
@@ -124,37 +128,29 @@ __global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeAr
     const uint16_t *Pg = a.cache.P;
     Tout *outp = static_cast<Tout *>(a.out);
 
-    // Loads only (no select on a loaded value): a token past the end reads the block's last token and
-    // is zeroed when the tile is built; factor rows beyond the rank are skipped by a uniform branch.
-    auto fetch = [&](long long blk, int tile, int rank) {
-        DtTileRegs<BITS> g;
-        const int tok = min(tile * 128 + r, n - 1);
-        const size_t t = static_cast<size_t>(blk) * n + tok;
-        {   // the token's row is 16 BITS bytes; this thread's 64 codes are its half `box`
-            const uint2 *src = reinterpret_cast<const uint2 *>(a.cache.codes + t * (16 * BITS) + 8 * BITS * box);
-#pragma unroll
-            for (int w = 0; w < BITS; ++w) {
-                const uint2 v = __ldg(src + w);
-                g.cw[2 * w] = v.x;
-                g.cw[2 * w + 1] = v.y;
-            }
-        }
-        g.rho = a.cache.norms[t];
-#pragma unroll
-        for (int i = 0; i < RMAX; ++i) {
-            g.p[i] = 0u;
-            if (i < rank) g.p[i] = Pg[(static_cast<size_t>(blk) * RMAX + i) * n + tok];
-        }
-        return g;
+    // One thread of the half asks the copy engine for the raw data of a tile (ranks are clamped to the
+    // rows the raw area holds; the library never stores more than the pilot k = 11).
+    constexpr uint32_t ROW = 16 * BITS;
+    uint8_t *raw = hbase + DT_H_RAW;
+    auto issue = [&](long long blk, int tile, int rank) {
+        const int tok0 = tile * 128;
+        const uint32_t rows = static_cast<uint32_t>(min(128, n - tok0));
+        const size_t t0 = static_cast<size_t>(blk) * n + tok0;
+        mbar_arrive_expect_tx(&raw_full[half], rows * (ROW + 2u) + static_cast<uint32_t>(rank) * rows * 2u);
+        dt_bulk_load(raw, a.cache.codes + t0 * ROW, rows * ROW, &raw_full[half]);
+        dt_bulk_load(raw + DT_RAW_NORMS, a.cache.norms + t0, rows * 2u, &raw_full[half]);
+        for (int i = 0; i < rank; ++i)
+            dt_bulk_load(raw + DT_RAW_P + i * 256, Pg + (static_cast<size_t>(blk) * RMAX + i) * n + tok0, rows * 2u, &raw_full[half]);
     };
 
-    uint32_t phase = 0;
+    uint32_t phase = 0, raw_phase = 0;
     bool alive = true, store_pending = false;
     const long long blk0 = 2ll * blockIdx.x + half, bstep = 2ll * gridDim.x;
-    int rank_next = (blk0 < a.nb) ? a.cache.rank[blk0] : 0;
+    int rank_next = (blk0 < a.nb) ? max(0, min(a.cache.rank[blk0], DT_PMAX)) : 0;
+    if (ht == 0 && blk0 < a.nb) issue(blk0, 0, rank_next);
     for (long long blk = blk0; blk < a.nb && alive; blk += bstep) {
-        const int rank = max(0, min(rank_next, RMAX));
-        if (blk + bstep < a.nb) rank_next = a.cache.rank[blk + bstep];   // known long before the next block starts
+        const int rank = rank_next;
+        if (blk + bstep < a.nb) rank_next = max(0, min(a.cache.rank[blk + bstep], DT_PMAX));   // known long before the next block starts
         {   // B operand of D2: row j, K = i: zeta_i[j] (zero beyond the rank); this thread: row r, entries 8 box .. 8 box + 7
             uint32_t vw[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
@@ -164,13 +160,34 @@ __global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeAr
             }
             *reinterpret_cast<uint4 *>(hbase + DT_H_V + dt_offset(r, box)) = make_uint4(vw[0], vw[1], vw[2], vw[3]);
         }
-        DtTileRegs<BITS> g = fetch(blk, 0, rank);
         for (int tile = 0; tile < tiles; ++tile) {
             const bool valid = tile * 128 + r < n;
+            // the tile's raw data (asked for one tile ago); rows past the end of the block were not copied
+            if (!mbar_wait(&raw_full[half], raw_phase, &abort_flag)) {
+                alive = false;
+                break;
+            }
+            raw_phase ^= 1u;
+            uint32_t cw[2 * BITS];
+#pragma unroll
+            for (int w = 0; w < BITS; ++w) {
+                const uint2 v = *reinterpret_cast<const uint2 *>(raw + r * ROW + 8 * BITS * box + 8 * w);
+                cw[2 * w] = valid ? v.x : 0u;
+                cw[2 * w + 1] = valid ? v.y : 0u;
+            }
+            const uint32_t rho_raw = valid ? *reinterpret_cast<const unsigned short *>(raw + DT_RAW_NORMS + 2 * r) : 0u;
+            uint32_t pw[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) pw[i] = 0u;
+            if (box == 0 && valid) {
+#pragma unroll
+                for (int i = 0; i < DT_PMAX; ++i)
+                    if (i < rank) pw[i >> 1] |= static_cast<uint32_t>(*reinterpret_cast<const unsigned short *>(raw + DT_RAW_P + i * 256 + 2 * r)) << (16 * (i & 1));
+            }
             {   // A operand of D1: this token's 64 coordinates of column half `box`, as fp16 centroids
                 uint32_t o[4][8];
 #pragma unroll
-                for (int q = 0; q < 4; ++q) expand16_codes<BITS>(g.cw, q, a.lo_tab, a.hi_tab, o[q]);
+                for (int q = 0; q < 4; ++q) expand16_codes<BITS>(cw, q, a.lo_tab, a.hi_tab, o[q]);
                 // the tile still holds the previous tile's output until the copy engine has read it: the
                 // expansion above ran in the shadow of that read
                 if (store_pending) {
@@ -184,14 +201,11 @@ __global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeAr
                     *reinterpret_cast<uint4 *>(hbase + DT_H_A + dt_offset(r, 8 * box + 2 * q + 1)) = make_uint4(o[q][4], o[q][5], o[q][6], o[q][7]);
                 }
                 if (box == 0) {   // A operand of D2: the token's factor entries
-                    uint32_t pw[8];
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) pw[i] = valid ? (g.p[2 * i] | (g.p[2 * i + 1] << 16)) : 0u;
                     *reinterpret_cast<uint4 *>(hbase + DT_H_P + dt_offset(r, 0)) = make_uint4(pw[0], pw[1], pw[2], pw[3]);
                     *reinterpret_cast<uint4 *>(hbase + DT_H_P + dt_offset(r, 1)) = make_uint4(pw[4], pw[5], pw[6], pw[7]);
                 }
             }
-            const float f = valid ? __half2float(__ushort_as_half(static_cast<unsigned short>(g.rho))) * a.inv_scale : 0.0f;
+            const float f = __half2float(__ushort_as_half(static_cast<unsigned short>(rho_raw))) * a.inv_scale;
             fence_proxy_async_smem();   // the operands were written by ordinary stores and are read by the tensor core
             dt_bar_sync(half);
             if (ht == 0) {
@@ -207,8 +221,10 @@ __global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeAr
                 }
                 umma_f16(d2, umma_desc_sw128(smem_u32(hbase + DT_H_P), 16, 1024), umma_desc_sw128(smem_u32(hbase + DT_H_V), 16, 1024), idesc, 0u);
                 umma_commit(&mma_done[half]);
+                // every thread has taken its part of the raw area (the barrier above): ask for the next tile
+                if (tile + 1 < tiles) issue(blk, tile + 1, rank);
+                else if (blk + bstep < a.nb) issue(blk + bstep, 0, rank_next);
             }
-            if (tile + 1 < tiles) g = fetch(blk, tile + 1, rank);   // behind the MMAs
             if (!mbar_wait(&mma_done[half], phase, &abort_flag)) {
                 alive = false;
                 break;
@@ -267,6 +283,10 @@ __global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeAr
         }
     }
 
+    if (!alive && ht == 0) {   // gave up with a copy of raw data possibly in flight: let it land before the CTA goes away
+        volatile int unused = 0;
+        mbar_wait(&raw_full[half], raw_phase, &unused);
+    }
     if (sizeof(Tout) == 2 && ht == 0) bulk_wait_all();
     __syncthreads();
     if (abort_flag && tid == 0) atomicOr(a.err, TC_ERR_DECODE_TIMEOUT);
@@ -279,8 +299,8 @@ __global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeAr
 float best_table_scale(const Codebook &cb, uint16_t (&table)[16]);
 
 bool decode_tc_supported(const eosq_cache_t &cache, int bits, const void *out_blocks) {
-    return (bits == 2 || bits == 3) && (reinterpret_cast<uintptr_t>(cache.codes) & 15u) == 0 &&
-           (reinterpret_cast<uintptr_t>(out_blocks) & 15u) == 0;
+    auto aligned = [](const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; };   // bulk copies and tensor stores
+    return (bits == 2 || bits == 3) && aligned(cache.codes) && aligned(cache.norms) && aligned(cache.P) && aligned(out_blocks);
 }
 
 template <typename Tout, int BITS>
