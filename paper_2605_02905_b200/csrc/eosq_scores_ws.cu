@@ -101,11 +101,16 @@ __global__ void __launch_bounds__(D) scores_w_kernel(const float *__restrict__ p
     float w[WS_NQ];
 #pragma unroll
     for (int g = 0; g < WS_NQ; ++g) w[g] = 0.0f;
-#pragma unroll 4
-    for (int j = 0; j < D; ++j) {
-        const float pv = __ldg(pi_t + j * D + c);
+#pragma unroll 1
+    for (int j0 = 0; j0 < D; j0 += 32) {
+        float pv[32];
 #pragma unroll
-        for (int g = 0; g < WS_NQ; ++g) w[g] = fmaf(pv, qs[g][j], w[g]);
+        for (int jj = 0; jj < 32; ++jj) pv[jj] = __ldg(pi_t + (j0 + jj) * D + c);   // 32 loads in flight: the kernel is all L2 latency
+#pragma unroll
+        for (int jj = 0; jj < 32; ++jj) {
+#pragma unroll
+            for (int g = 0; g < WS_NQ; ++g) w[g] = fmaf(pv[jj], qs[g][j0 + jj], w[g]);
+        }
     }
     uint8_t *img = wimg + static_cast<size_t>(hd) * 4096;
 #pragma unroll
