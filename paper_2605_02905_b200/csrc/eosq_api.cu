@@ -89,7 +89,7 @@ cudaEvent_t take_event(eosq_ctx *ctx) {
     return e;
 }
 
-// Runs `launch` (which enqueues exactly one kernel on `s`), counting it and, when profiling is
+// Runs `launch` (which enqueues one kernel on `s`; the score path adds its extra ones itself), counting it and, when profiling is
 // on, bracketing it with events.
 template <typename F>
 void run_stage(eosq_ctx *ctx, int stage, cudaStream_t s, F &&launch) {
@@ -321,11 +321,13 @@ extern "C" int eosq_scores(eosq_ctx *ctx, const eosq_cache_t *kcache, int64_t nu
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     if (scores_tc_supported(*kcache, bits, n) && (reinterpret_cast<uintptr_t>(kcache->codes) & 15u) == 0) {
         bool setup_ok = true;
+        int64_t kernels = 0;
         run_stage(ctx, ST_SCORES, s, [&] {
             setup_ok = launch_scores_tc(*kcache, num_kv_heads, blocks_per_head, head_stride_blocks, n, rot, cb,
                                         static_cast<const __half *>(q), G, scale, scores, ctx->dev_err, ctx->sm_count, &ctx->scores_w,
-                                        &ctx->scores_w_bytes, s);
+                                        &ctx->scores_w_bytes, &kernels, s);
         });
+        ctx->launches += std::max<int64_t>(kernels, 1) - 1;   // run_stage counted one
         if (!setup_ok) {
             ctx->last_error = "tensor-core score kernel: launch set-up failed";
             return EOSQ_ERR_CUDA;

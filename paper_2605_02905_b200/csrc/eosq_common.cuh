@@ -159,7 +159,7 @@ void launch_scores_plain(const eosq_cache_t &cache, int64_t heads, int64_t bph, 
 bool scores_tc_supported(const eosq_cache_t &cache, int bits, int n);
 bool launch_scores_tc(const eosq_cache_t &cache, int64_t heads, int64_t bph, int64_t head_stride, int n, const Rotation &rot,
                       const Codebook &cb, const __half *q, int G, float scale, float *scores, int *err, int sm_count,
-                      void **scratch, size_t *scratch_bytes, cudaStream_t s);
+                      void **scratch, size_t *scratch_bytes, int64_t *kernels, cudaStream_t s);
 
 // ---- small device helpers -------------------------------------------------------------------
 __device__ __forceinline__ double warp_sum(double v) {

@@ -329,7 +329,7 @@ float best_table_scale(const Codebook &cb, uint16_t (&table)[16]) {
 bool scores_ws_supported(const eosq_cache_t &cache, int bits, int n);
 bool launch_scores_ws(const eosq_cache_t &cache, int bits, int64_t heads, int64_t bph, int64_t head_stride, int n, const Rotation &rot,
                       const uint16_t (&table)[16], float kappa, const __half *q, int G, float scale, float *scores, int *err,
-                      int sm_count, void **scratch, size_t *scratch_bytes, cudaStream_t s);
+                      int sm_count, void **scratch, size_t *scratch_bytes, int64_t *kernels, cudaStream_t s);
 
 // 2-bit codes always (the simpler kernel below takes what the warp-specialised one cannot); 3-bit codes
 // where the warp-specialised kernel applies.
@@ -339,7 +339,7 @@ bool scores_tc_supported(const eosq_cache_t &cache, int bits, int n) {
 
 bool launch_scores_tc(const eosq_cache_t &cache, int64_t heads, int64_t bph, int64_t head_stride, int n, const Rotation &rot,
                       const Codebook &cb, const __half *q, int G, float scale, float *scores, int *err, int sm_count,
-                      void **scratch, size_t *scratch_bytes, cudaStream_t s) {
+                      void **scratch, size_t *scratch_bytes, int64_t *kernels, cudaStream_t s) {
     static bool configured = false;
     constexpr size_t smem = 24576 + 1024;
     if (!configured) {
@@ -356,7 +356,7 @@ bool launch_scores_tc(const eosq_cache_t &cache, int64_t heads, int64_t bph, int
     const float kappa = kappas[cb.bits];
     if (scores_ws_supported(cache, cb.bits, n))
         return launch_scores_ws(cache, cb.bits, heads, bph, head_stride, n, rot, table, kappa, q, G, scale, scores, err, sm_count, scratch,
-                                scratch_bytes, s);
+                                scratch_bytes, kernels, s);
     if (cb.bits != 2) return false;
     ScoresArgs a;
     a.cache = cache;
@@ -381,6 +381,7 @@ bool launch_scores_tc(const eosq_cache_t &cache, int64_t heads, int64_t bph, int
     for (int g0 = 0; g0 < G; g0 += SC_NQ) {
         a.g0 = g0;
         scores_tc_kernel<<<grid, SC_THREADS, smem, s>>>(a);
+        *kernels += 1;
     }
     return true;
 }

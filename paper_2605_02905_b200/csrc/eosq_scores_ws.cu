@@ -526,7 +526,7 @@ bool scores_ws_supported(const eosq_cache_t &cache, int bits, int n) {
 
 template <int BITS>
 static bool launch_scores_ws_as(WsArgs &a, int G, int grid, const CUtensorMap &m4, const CUtensorMap &m8, const CUtensorMap &m12,
-                                const float *pi_t, uint8_t *wimg, cudaStream_t s) {
+                                const float *pi_t, uint8_t *wimg, int64_t *kernels, cudaStream_t s) {
     static bool configured = false;
     if (!configured) {
         if (cudaFuncSetAttribute(scores_ws_kernel<BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -538,13 +538,14 @@ static bool launch_scores_ws_as(WsArgs &a, int G, int grid, const CUtensorMap &m
         a.g0 = g0;
         scores_w_kernel<<<a.heads, D, 0, s>>>(pi_t, a.q, G, g0, wimg);
         scores_ws_kernel<BITS><<<grid, WS_THREADS, WsLayout<BITS>::SMEM_BYTES, s>>>(a, m4, m8, m12);
+        *kernels += 2;
     }
     return true;
 }
 
 bool launch_scores_ws(const eosq_cache_t &cache, int bits, int64_t heads, int64_t bph, int64_t head_stride, int n, const Rotation &rot,
                       const uint16_t (&table)[16], float kappa, const __half *q, int G, float scale, float *scores, int *err,
-                      int sm_count, void **scratch, size_t *scratch_bytes, cudaStream_t s) {
+                      int sm_count, void **scratch, size_t *scratch_bytes, int64_t *kernels, cudaStream_t s) {
     if (heads * bph > 0x7fffffff || head_stride > 0x7fffffff || (bits != 2 && bits != 3)) return false;
     WsArgs a;
     a.cache = cache;
@@ -581,8 +582,8 @@ bool launch_scores_ws(const eosq_cache_t &cache, int bits, int64_t heads, int64_
         !make_factor_tensor_map(cache.P, nb_total, n, 12, &m12))
         return false;
     uint8_t *wimg = static_cast<uint8_t *>(*scratch);
-    return bits == 2 ? launch_scores_ws_as<2>(a, G, grid, m4, m8, m12, rot.pi_t, wimg, s)
-                     : launch_scores_ws_as<3>(a, G, grid, m4, m8, m12, rot.pi_t, wimg, s);
+    return bits == 2 ? launch_scores_ws_as<2>(a, G, grid, m4, m8, m12, rot.pi_t, wimg, kernels, s)
+                     : launch_scores_ws_as<3>(a, G, grid, m4, m8, m12, rot.pi_t, wimg, kernels, s);
 }
 
 }  // namespace eosq
