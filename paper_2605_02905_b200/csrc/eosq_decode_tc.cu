@@ -1,4 +1,4 @@
-// Tensor-core decode for 2- and 3-bit codes (Algorithm 1 DeQuant + the stored low-rank part):
+// Tensor-core decode for 1- to 4-bit codes (Algorithm 1 DeQuant + the stored low-rank part):
 //   x_t = rho_t (z_t Pi) + sum_i P[t][i] zeta_i,     z_t = centroids of the codes of token t.
 //
 // One persistent CTA of 512 threads per SM holds the rotation once, as the B operand of
@@ -32,13 +32,13 @@ constexpr uint32_t DT_OFF_PI_HI = 0, DT_OFF_PI_LO = 2 * DT_BOX;
 constexpr uint32_t DT_OFF_HALF = 4 * DT_BOX;          // per half: A tile (2 boxes), factor tile (1 box), right vectors (1 box)
 constexpr uint32_t DT_H_A = 0, DT_H_P = 2 * DT_BOX, DT_H_V = 3 * DT_BOX;
 // ... and the raw data of the next tile, copied in while the current one is worked on: packed codes
-// (128 tokens x up to 48 bytes), norms, up to 12 factor rows of 128 fp16
+// (128 tokens x 16 BITS bytes), norms, up to 12 factor rows of 128 fp16
 constexpr int DT_PMAX = 12;
-constexpr uint32_t DT_H_RAW = 4 * DT_BOX, DT_RAW_NORMS = 128 * 48, DT_RAW_P = DT_RAW_NORMS + 256;
-constexpr uint32_t DT_RAW_BYTES = 10240;
-static_assert(DT_RAW_P + DT_PMAX * 256 <= DT_RAW_BYTES && KPILOT < DT_PMAX, "the raw area holds one tile");
+constexpr uint32_t DT_H_RAW = 4 * DT_BOX;
+constexpr uint32_t DT_RAW_BYTES = 12288;
+static_assert(128 * 64 + 256 + DT_PMAX * 256 <= DT_RAW_BYTES && KPILOT < DT_PMAX, "the raw area holds one tile of 4-bit codes");
 constexpr uint32_t DT_HALF_BYTES = 4 * DT_BOX + DT_RAW_BYTES;
-constexpr size_t DT_SMEM = DT_OFF_HALF + 2 * DT_HALF_BYTES + 1024;   // 213 KB
+constexpr size_t DT_SMEM = DT_OFF_HALF + 2 * DT_HALF_BYTES + 1024;   // 217 KB
 constexpr uint32_t DT_TMEM_COLS = 512;                // per half: D1 128 columns, D2 128 columns
 
 // Byte offset of the 16-byte chunk `jc` (8 fp16 of K) of row `row` in a K-major, 128-byte-swizzled
@@ -55,7 +55,7 @@ struct DecodeArgs {
     eosq_cache_t cache;
     int nb, n;
     float inv_scale;            // 1 / (kappa 2^12)
-    uint32_t lo_tab[2], hi_tab[2];   // low / high bytes of the fp16 centroids times kappa (level k in byte k)
+    uint32_t lo_tab[4], hi_tab[4];   // low / high bytes of the fp16 centroids times kappa (level k in byte k)
     const float *pi_t;          // pi_t[j][c] = Pi[c][j]
     void *out;
     int *err;
@@ -74,7 +74,7 @@ bool make_block_tensor_map(const void *blocks, int64_t nb, int n, CUtensorMap *o
 // 128-byte swizzled - the layout of the A tile, which doubles as the staging buffer of the stores.
 template <typename Tout, int BITS>
 __global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeArgs a, const __grid_constant__ CUtensorMap omap) {
-    static_assert(BITS == 2 || BITS == 3, "byte-permute expansion covers up to eight levels");
+    static_assert(BITS >= 1 && BITS <= 4, "code widths of the format");
     extern __shared__ uint8_t dt_smem_raw[];
     __shared__ __align__(8) uint64_t mma_done[2], raw_full[2];
     __shared__ uint32_t tmem_base_s;
@@ -130,7 +130,7 @@ __global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeAr
 
     // One thread of the half asks the copy engine for the raw data of a tile (ranks are clamped to the
     // rows the raw area holds; the library never stores more than the pilot k = 11).
-    constexpr uint32_t ROW = 16 * BITS;
+    constexpr uint32_t ROW = 16 * BITS, DT_RAW_NORMS = 128 * ROW, DT_RAW_P = DT_RAW_NORMS + 256;
     uint8_t *raw = hbase + DT_H_RAW;
     auto issue = [&](long long blk, int tile, int rank) {
         const int tok0 = tile * 128;
@@ -300,7 +300,7 @@ float best_table_scale(const Codebook &cb, uint16_t (&table)[16]);
 
 bool decode_tc_supported(const eosq_cache_t &cache, int bits, const void *out_blocks) {
     auto aligned = [](const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; };   // bulk copies and tensor stores
-    return (bits == 2 || bits == 3) && aligned(cache.codes) && aligned(cache.norms) && aligned(cache.P) && aligned(out_blocks);
+    return bits >= 1 && bits <= 4 && aligned(cache.codes) && aligned(cache.norms) && aligned(cache.P) && aligned(out_blocks);
 }
 
 template <typename Tout, int BITS>
@@ -321,14 +321,14 @@ bool launch_decode_tc(const eosq_cache_t &cache, int64_t nb, int n, const Rotati
     static uint16_t table[5][16];
     static float kappa[5] = {0.0f, 0.0f, 0.0f, 0.0f, 0.0f};
     const int bits = cb.bits;
-    if (bits != 2 && bits != 3) return false;
+    if (bits < 1 || bits > 4) return false;
     if (kappa[bits] == 0.0f) kappa[bits] = best_table_scale(cb, table[bits]);
     DecodeArgs a;
     a.cache = cache;
     a.nb = static_cast<int>(nb);
     a.n = n;
     a.inv_scale = 1.0f / (kappa[bits] * DT_PSCALE);
-    a.lo_tab[0] = a.lo_tab[1] = a.hi_tab[0] = a.hi_tab[1] = 0u;
+    for (int w = 0; w < 4; ++w) a.lo_tab[w] = a.hi_tab[w] = 0u;
     for (int k = 0; k < (1 << bits); ++k) {
         a.lo_tab[k >> 2] |= static_cast<uint32_t>(table[bits][k] & 0xFFu) << (8 * (k & 3));
         a.hi_tab[k >> 2] |= static_cast<uint32_t>(table[bits][k] >> 8) << (8 * (k & 3));
@@ -339,10 +339,21 @@ bool launch_decode_tc(const eosq_cache_t &cache, int64_t nb, int n, const Rotati
     const int grid = static_cast<int>(std::min<int64_t>((nb + 1) / 2, sm_count));
     CUtensorMap omap;
     std::memset(&omap, 0, sizeof(omap));
-    if (out_dtype == EOSQ_F32)
-        return bits == 2 ? launch_decode_tc_as<float, 2>(a, omap, grid, s) : launch_decode_tc_as<float, 3>(a, omap, grid, s);
+    if (out_dtype == EOSQ_F32) {
+        switch (bits) {
+            case 1: return launch_decode_tc_as<float, 1>(a, omap, grid, s);
+            case 2: return launch_decode_tc_as<float, 2>(a, omap, grid, s);
+            case 3: return launch_decode_tc_as<float, 3>(a, omap, grid, s);
+            default: return launch_decode_tc_as<float, 4>(a, omap, grid, s);
+        }
+    }
     if (!make_block_tensor_map(out_blocks, nb, n, &omap)) return false;
-    return bits == 2 ? launch_decode_tc_as<__half, 2>(a, omap, grid, s) : launch_decode_tc_as<__half, 3>(a, omap, grid, s);
+    switch (bits) {
+        case 1: return launch_decode_tc_as<__half, 1>(a, omap, grid, s);
+        case 2: return launch_decode_tc_as<__half, 2>(a, omap, grid, s);
+        case 3: return launch_decode_tc_as<__half, 3>(a, omap, grid, s);
+        default: return launch_decode_tc_as<__half, 4>(a, omap, grid, s);
+    }
 }
 
 }  // namespace eosq

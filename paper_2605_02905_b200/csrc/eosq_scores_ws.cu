@@ -54,7 +54,7 @@ struct WsArgs {
     int bph, head_stride, heads;   // blocks per head, block stride between heads, heads
     int n, G, g0;
     float scale, inv_code;
-    uint32_t lo_tab[2], hi_tab[2];   // low / high bytes of the fp16 centroids times kappa (level k in byte k)
+    uint32_t lo_tab[4], hi_tab[4];   // low / high bytes of the fp16 centroids times kappa (level k in byte k)
     const uint8_t *wimg;   // per head: the 4096-byte image of the operand W = Pi q (made by scores_w_kernel)
     const __half *q;
     float *scores;
@@ -556,7 +556,7 @@ bool launch_scores_ws(const eosq_cache_t &cache, int bits, int64_t heads, int64_
     a.G = G;
     a.scale = scale;
     a.inv_code = 1.0f / (kappa * WS_QSCALE);
-    a.lo_tab[0] = a.lo_tab[1] = a.hi_tab[0] = a.hi_tab[1] = 0u;
+    for (int w = 0; w < 4; ++w) a.lo_tab[w] = a.hi_tab[w] = 0u;
     for (int k = 0; k < (1 << bits); ++k) {
         a.lo_tab[k >> 2] |= static_cast<uint32_t>(table[k] & 0xFFu) << (8 * (k & 3));
         a.hi_tab[k >> 2] |= static_cast<uint32_t>(table[k] >> 8) << (8 * (k & 3));
