@@ -331,10 +331,10 @@ bool launch_scores_ws(const eosq_cache_t &cache, int bits, int64_t heads, int64_
                       const uint16_t (&table)[16], float kappa, const __half *q, int G, float scale, float *scores, int *err,
                       int sm_count, void **scratch, size_t *scratch_bytes, int64_t *kernels, cudaStream_t s);
 
-// 2-bit codes always (the simpler kernel below takes what the warp-specialised one cannot); 3-bit codes
-// where the warp-specialised kernel applies.
+// 2-bit codes always (the simpler kernel below takes what the warp-specialised one cannot); the other
+// widths where the warp-specialised kernel applies.
 bool scores_tc_supported(const eosq_cache_t &cache, int bits, int n) {
-    return n >= 128 && (bits == 2 || (bits == 3 && scores_ws_supported(cache, bits, n)));
+    return n >= 128 && (bits == 2 || scores_ws_supported(cache, bits, n));
 }
 
 bool launch_scores_tc(const eosq_cache_t &cache, int64_t heads, int64_t bph, int64_t head_stride, int n, const Rotation &rot,

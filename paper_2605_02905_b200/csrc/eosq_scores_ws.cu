@@ -1,4 +1,4 @@
-// Warp-specialised attention-logit kernel for 2- and 3-bit codes (Remark 6.4): one persistent CTA of 16
+// Warp-specialised attention-logit kernel for 1- to 4-bit codes (Remark 6.4): one persistent CTA of 16
 // warps per SM in which loading, code expansion, the MMAs and the output run concurrently on
 // different tiles.
 //
@@ -27,7 +27,7 @@ constexpr int TC_ERR_SCORES_WS_TIMEOUT = 8;
 
 constexpr int WS_THREADS = 512;
 constexpr int WS_NQ = 8;                   // query vectors per pass
-constexpr int WS_STAGES = 5;               // shared-memory stages of WS_TPS tiles each
+constexpr int WS_STAGES = 5;               // shared-memory stages of WS_TPS tiles each (four with 4-bit codes: their stages are larger)
 constexpr int WS_TPS = 4;                  // tiles per stage: few large copies keep the copy engine's queue short
 constexpr int WS_BUFS = 4;
 constexpr int WS_PMAX = 12;                // factor rows staged per tile (rank <= pilot k = 11)
@@ -36,9 +36,10 @@ constexpr uint32_t WS_ST_CODES = 0;
 constexpr uint32_t WS_ST_PBOX = WS_PMAX * 512;
 template <int BITS> struct WsLayout {
     static constexpr uint32_t ROW = 16 * BITS;                              // code bytes per token
+    static constexpr int STAGES = (BITS == 4) ? WS_STAGES - 1 : WS_STAGES;
     static constexpr uint32_t ST_NORMS = 512 * ROW, ST_P = ST_NORMS + 1024;
     static constexpr uint32_t STAGE_BYTES = ST_P + 2 * WS_ST_PBOX;         // 29696 (2 bits), 37888 (3 bits)
-    static constexpr uint32_t OFF_B1 = WS_STAGES * STAGE_BYTES;            // 2 x 4096: W, hi rows 0-7, lo rows 8-15
+    static constexpr uint32_t OFF_B1 = STAGES * STAGE_BYTES;            // 2 x 4096: W, hi rows 0-7, lo rows 8-15
     static constexpr uint32_t OFF_B2 = OFF_B1 + 2 * 4096;                  // 2 x 2048: Aq
     static constexpr uint32_t OFF_V = OFF_B2 + 2 * 2048;                   // 2 x 4096: right vectors (fp16)
     static constexpr uint32_t OFF_Q = OFF_V + 2 * 4096;                    // 2 x (8 x 128) fp32 queries, by head parity
@@ -197,13 +198,13 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
                 }
                 alive = __shfl_sync(0xffffffffu, alive, 0);
                 for (int tile = 0; tile < tiles && alive; tile += WS_TPS, ++sseq) {
-                    const int stage = sseq % WS_STAGES;
+                    const int stage = sseq % L::STAGES;
                     const int tok0 = tile * 128;
                     const uint32_t rows = static_cast<uint32_t>(min(128 * WS_TPS, n - tok0));
                     const uint32_t boxes = (rows + 255u) >> 8;
                     const int r4 = (rank + 3) >> 2;
                     if (lane == 0) {
-                        alive = mbar_wait(&bars.st_empty[stage], ((sseq / WS_STAGES) & 1u) ^ 1u, &abort_flag);
+                        alive = mbar_wait(&bars.st_empty[stage], ((sseq / L::STAGES) & 1u) ^ 1u, &abort_flag);
                         if (alive) {
                             st_rank[stage] = rank;
                             mbar_arrive_expect_tx(&bars.st_full[stage], rows * (L::ROW + 2u) + boxes * static_cast<uint32_t>(r4) * 2048u);
@@ -388,8 +389,8 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
             for (int tile = 0; tile < tiles; ++tile, ++seq) {
                 if (static_cast<int>(seq & 1u) != grp) continue;
                 const uint32_t sseq = sbase + tile / WS_TPS;
-                const int stage = sseq % WS_STAGES, buf = seq & (WS_BUFS - 1);
-                if (!mbar_wait(&bars.st_full[stage], (sseq / WS_STAGES) & 1u, &abort_flag)) {
+                const int stage = sseq % L::STAGES, buf = seq & (WS_BUFS - 1);
+                if (!mbar_wait(&bars.st_full[stage], (sseq / L::STAGES) & 1u, &abort_flag)) {
                     alive = false;
                     break;
                 }
@@ -521,7 +522,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
 
 bool scores_ws_supported(const eosq_cache_t &cache, int bits, int n) {
     auto aligned = [](const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; };
-    return (bits == 2 || bits == 3) && n >= 128 && (n % 8) == 0 && aligned(cache.codes) && aligned(cache.norms) && aligned(cache.P) && aligned(cache.V);
+    return bits >= 1 && bits <= 4 && n >= 128 && (n % 8) == 0 && aligned(cache.codes) && aligned(cache.norms) && aligned(cache.P) && aligned(cache.V);
 }
 
 template <int BITS>
@@ -546,7 +547,7 @@ static bool launch_scores_ws_as(WsArgs &a, int G, int grid, const CUtensorMap &m
 bool launch_scores_ws(const eosq_cache_t &cache, int bits, int64_t heads, int64_t bph, int64_t head_stride, int n, const Rotation &rot,
                       const uint16_t (&table)[16], float kappa, const __half *q, int G, float scale, float *scores, int *err,
                       int sm_count, void **scratch, size_t *scratch_bytes, int64_t *kernels, cudaStream_t s) {
-    if (heads * bph > 0x7fffffff || head_stride > 0x7fffffff || (bits != 2 && bits != 3)) return false;
+    if (heads * bph > 0x7fffffff || head_stride > 0x7fffffff || bits < 1 || bits > 4) return false;
     WsArgs a;
     a.cache = cache;
     a.bph = static_cast<int>(bph);
@@ -582,8 +583,12 @@ bool launch_scores_ws(const eosq_cache_t &cache, int bits, int64_t heads, int64_
         !make_factor_tensor_map(cache.P, nb_total, n, 12, &m12))
         return false;
     uint8_t *wimg = static_cast<uint8_t *>(*scratch);
-    return bits == 2 ? launch_scores_ws_as<2>(a, G, grid, m4, m8, m12, rot.pi_t, wimg, kernels, s)
-                     : launch_scores_ws_as<3>(a, G, grid, m4, m8, m12, rot.pi_t, wimg, kernels, s);
+    switch (bits) {
+        case 1: return launch_scores_ws_as<1>(a, G, grid, m4, m8, m12, rot.pi_t, wimg, kernels, s);
+        case 2: return launch_scores_ws_as<2>(a, G, grid, m4, m8, m12, rot.pi_t, wimg, kernels, s);
+        case 3: return launch_scores_ws_as<3>(a, G, grid, m4, m8, m12, rot.pi_t, wimg, kernels, s);
+        default: return launch_scores_ws_as<4>(a, G, grid, m4, m8, m12, rot.pi_t, wimg, kernels, s);
+    }
 }
 
 }  // namespace eosq
