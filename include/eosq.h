@@ -163,6 +163,10 @@ int eosq_encode_static(eosq_ctx *ctx, const void *blocks, int in_dtype, int64_t 
  * Reconstruct blocks from a compressed cache (Algorithm 1 last TQ_MSE line, Algorithm 2 Return):
  *   x_hat[t] = sum_{i<r} P[i][t] V[i][:] + norms[t] * Pi^T centroids[codes[t]].
  *   out_blocks dev [num_blocks][n][d] of out_dtype (EOSQ_F16 or EOSQ_F32).
+ * With codes, norms, P and out_blocks 16-byte aligned the tensor-core kernel runs; it (and the score
+ * kernel) reads at most 12 factor rows per block (eosq_encode stores at most the pilot k = 11), so a
+ * cache written elsewhere with a larger rank word is truncated to 12.  Other layouts take a slower
+ * CUDA-core kernel.
  */
 int eosq_decode(eosq_ctx *ctx, const eosq_cache_t *cache, int64_t num_blocks, int n, int d, int bits,
                 uint64_t seed, void *out_blocks, int out_dtype, void *cuda_stream);
