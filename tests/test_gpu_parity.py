@@ -235,14 +235,15 @@ def test_nonfinite_input_is_flagged_not_fatal(ctx):
     assert eosq.eosq_check_status(ctx, cache) == 1
 
 
-def test_full_size_cache_sampled_blocks(ctx):
-    """Config 2 in the benchmark's launch configuration: the whole Llama-3.1-8B-shaped 32k cache
-    (16384 blocks, 4 GiB) is encoded in one call; sampled blocks go to the oracle one by one, and
-    properties that hold at any size are checked on everything."""
+@pytest.mark.parametrize("bits", [2, 3])
+def test_full_size_cache_sampled_blocks(ctx, bits):
+    """Config 2 in the benchmark's launch configuration (both of its code widths): the whole
+    Llama-3.1-8B-shaped 32k cache (16384 blocks, 4 GiB) is encoded, scored and decoded in one call each;
+    sampled blocks go to the oracle one by one, and properties that hold at any size are checked on everything."""
     w = synth.llama_32k(device="cuda")
     B = w.blocks.shape[0]
     assert B == 16384
-    cache = eosq.eosq_encode(ctx, w.blocks, 2, SEED)
+    cache = eosq.eosq_encode(ctx, w.blocks, bits, SEED)
     torch.cuda.synchronize()
     assert eosq.eosq_check_status(ctx, cache) == 0
     ranks = cache.rank
@@ -255,15 +256,22 @@ def test_full_size_cache_sampled_blocks(ctx):
     assert torch.allclose(eig[:256].sum(dim=1), fro, rtol=2e-3)
     pick = [0, 31, 32, 4097, 9000, B - 1]
     sub = w.blocks[pick].cpu()
-    sub_cache = eosq.Cache.allocate(len(pick), w.n, w.d, 2)
+    sub_cache = eosq.Cache.allocate(len(pick), w.n, w.d, bits)
     for name in ("codes", "norms", "rank", "sigma", "phi", "P", "V", "status", "eig", "lambda_plus", "vr32", "coef"):
         getattr(sub_cache, name).copy_(getattr(cache, name)[pick])
-    rep, enc = parity.compare_encode(sub, sub_cache, 2, SEED)
-    _report("llama_32k_sampled", rep)
+    rep, enc = parity.compare_encode(sub, sub_cache, bits, SEED)
+    _report(f"llama_32k_sampled_b{bits}", rep)
     assert rep["e2e_out_band_fraction"] < 1e-4
     # scores over the keys of the first layers, sampled (head, block) pairs against the oracle
     heads, bph, G = 16, 32, 4
     q = synth.queries(heads, G, seed=8).cuda()
     s = eosq.eosq_scores(ctx, cache, q, heads, bph, 2 * bph, SEED)
     torch.cuda.synchronize()
-    parity.compare_scores(cache, q, s, heads, bph, 2 * bph, 2, SEED, 1.0 / math.sqrt(128), pairs=[(0, 0), (5, 17), (15, 31)])
+    parity.compare_scores(cache, q, s, heads, bph, 2 * bph, bits, SEED, 1.0 / math.sqrt(128), pairs=[(0, 0), (5, 17), (15, 31)])
+    # decode of the whole cache to fp16; the sampled blocks against the oracle's decode of the same stored bytes
+    del s
+    dec = eosq.eosq_decode(ctx, cache, SEED, out_dtype=torch.float16)
+    torch.cuda.synchronize()
+    assert eosq.eosq_check_status(ctx, cache) == 0
+    assert torch.all(torch.isfinite(dec[::257].float()))
+    parity.compare_decode(sub_cache, dec[pick], bits, SEED, tol=1e-3)
