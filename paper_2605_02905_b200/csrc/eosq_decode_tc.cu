@@ -128,26 +128,33 @@ __global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeAr
     const uint16_t *Pg = a.cache.P;
     Tout *outp = static_cast<Tout *>(a.out);
 
-    // One thread of the half asks the copy engine for the raw data of a tile (ranks are clamped to the
-    // rows the raw area holds; the library never stores more than the pilot k = 11).
+    // The second warp of the half asks the copy engine for the raw data of a tile, one copy per lane (a
+    // thread needs over 100 cycles per copy it issues, and the first warp's lane 0 is busy issuing MMAs).
+    // Ranks are clamped to the rows the raw area holds; the library never stores more than the pilot k = 11.
     constexpr uint32_t ROW = 16 * BITS, DT_RAW_NORMS = 128 * ROW, DT_RAW_P = DT_RAW_NORMS + 256;
     uint8_t *raw = hbase + DT_H_RAW;
+    const int cl = ht - 32;   // lane of the copying warp
     auto issue = [&](long long blk, int tile, int rank) {
         const int tok0 = tile * 128;
         const uint32_t rows = static_cast<uint32_t>(min(128, n - tok0));
         const size_t t0 = static_cast<size_t>(blk) * n + tok0;
-        mbar_arrive_expect_tx(&raw_full[half], rows * (ROW + 2u) + static_cast<uint32_t>(rank) * rows * 2u);
-        dt_bulk_load(raw, a.cache.codes + t0 * ROW, rows * ROW, &raw_full[half]);
-        dt_bulk_load(raw + DT_RAW_NORMS, a.cache.norms + t0, rows * 2u, &raw_full[half]);
-        for (int i = 0; i < rank; ++i)
+        if (cl == 0) mbar_arrive_expect_tx(&raw_full[half], rows * (ROW + 2u) + static_cast<uint32_t>(rank) * rows * 2u);
+        __syncwarp();   // the byte count is announced before any copy can report completion
+        if (cl == 0) {
+            dt_bulk_load(raw, a.cache.codes + t0 * ROW, rows * ROW, &raw_full[half]);
+        } else if (cl == 1) {
+            dt_bulk_load(raw + DT_RAW_NORMS, a.cache.norms + t0, rows * 2u, &raw_full[half]);
+        } else if (cl - 2 < rank) {
+            const int i = cl - 2;
             dt_bulk_load(raw + DT_RAW_P + i * 256, Pg + (static_cast<size_t>(blk) * RMAX + i) * n + tok0, rows * 2u, &raw_full[half]);
+        }
     };
 
     uint32_t phase = 0, raw_phase = 0;
     bool alive = true, store_pending = false;
     const long long blk0 = 2ll * blockIdx.x + half, bstep = 2ll * gridDim.x;
     int rank_next = (blk0 < a.nb) ? max(0, min(a.cache.rank[blk0], DT_PMAX)) : 0;
-    if (ht == 0 && blk0 < a.nb) issue(blk0, 0, rank_next);
+    if (ht >= 32 && ht < 64 && blk0 < a.nb) issue(blk0, 0, rank_next);
     for (long long blk = blk0; blk < a.nb && alive; blk += bstep) {
         const int rank = rank_next;
         if (blk + bstep < a.nb) rank_next = max(0, min(a.cache.rank[blk + bstep], DT_PMAX));   // known long before the next block starts
@@ -221,6 +228,7 @@ __global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeAr
                 }
                 umma_f16(d2, umma_desc_sw128(smem_u32(hbase + DT_H_P), 16, 1024), umma_desc_sw128(smem_u32(hbase + DT_H_V), 16, 1024), idesc, 0u);
                 umma_commit(&mma_done[half]);
+            } else if (ht >= 32 && ht < 64) {
                 // every thread has taken its part of the raw area (the barrier above): ask for the next tile
                 if (tile + 1 < tiles) issue(blk, tile + 1, rank);
                 else if (blk + bstep < a.nb) issue(blk + bstep, 0, rank_next);
