@@ -52,7 +52,7 @@ constexpr size_t WS_PER_BLOCK = sizeof(double) * (D * D + 4 * D) + sizeof(float)
 // about 1e-8 of the largest eigenvalue, which would move smaller singular values by more than
 // 5e-5 relative.
 constexpr double REDO_RATIO = 1e-4;
-constexpr int64_t CHUNK_BLOCKS = 592;  // 4 per SM on 148 SMs: the scratch of one chunk stays L2 sized
+constexpr int64_t CHUNK_BLOCKS = 1184;  // 8 per SM on 148 SMs: what the second tridiagonalisation kernel can hold in flight
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -131,8 +131,8 @@ constexpr int64_t LIST_GRID = 148;
 inline unsigned list_grid(int64_t nb, const int *list) {
     return static_cast<unsigned>(list ? (nb < LIST_GRID ? nb : LIST_GRID) : nb);
 }
-constexpr int TRIDIAG_PARTS = 3;
-void launch_tridiag(int part, int64_t nb, const Workspace &ws, const int *list, const int *count, cudaStream_t s);
+constexpr int TRIDIAG_PARTS = 2;
+void launch_tridiag(int part, int64_t nb, const Workspace &ws, const int *list, const int *count, int sm_count, cudaStream_t s);
 // All eigenvalues of each tridiagonal matrix by Sturm bisection.
 void launch_eigvals(int64_t nb, const Workspace &ws, const int *list, const int *count, int *mark_list, cudaStream_t s);
 // Clears the redo list / appends every block whose eigenvalue range exceeds 1 / REDO_RATIO.

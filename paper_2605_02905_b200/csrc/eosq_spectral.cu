@@ -10,309 +10,6 @@
 namespace eosq {
 
 // ------------------------------------------------------------------------------------------
-// Householder tridiagonalisation with the matrix resident in registers as 8 x 8 cyclic tiles on a
-// G x G thread grid: thread (tr, tc) = (tid / G, tid % G) holds A[tr + G a][tc + G b], a, b < 8,
-// so every thread keeps an equal share of the shrinking trailing matrix, and a vector entry
-// fetched from shared memory feeds eight multiply-adds.
-//
-// Step k reflects with H = I - gamma u u^T, u = (0, .., 0, alpha - beta, A[k][k+2], .., A[k][N-1]),
-// alpha = A[k][k+1], beta = -sign(alpha) ||A[k][k+1..]||, gamma = 1 / (beta (beta - alpha)):
-//     p = gamma A u,  2K = gamma (u.p),  A <- A - u p^T - (p - 2K u) u^T.
-// u and p travel through shared memory (double buffered by the parity of k, two block-wide
-// barriers per step) in a permuted order that makes a thread's eight columns contiguous.
-//
-// Every step is a chain of dependent latencies (two barriers, a square root and a division, a
-// butterfly reduction), so one matrix cannot fill an SM.  The work is therefore split in two
-// kernels.  The head (G = 16, 256 threads, one CTA per SM) takes the 128 x 128 matrix through its
-// first 64 steps and leaves the 64 x 64 trailing matrix in the lower left quadrant of the matrix
-// in global memory, which no reflector uses.  The tail (G = 8, 64 threads) finishes that trailing
-// matrix with four CTAs per SM, whose latency chains overlap.  Row k of the matrix in global
-// memory receives u of step k, tau[k] receives gamma.
-// ------------------------------------------------------------------------------------------
-constexpr int TD_PSTRIDE = 10;   // doubles per column group in the permuted vectors (8 used, 2 pad)
-
-template <int G>
-__device__ __forceinline__ int td_pos(int j) {
-    return (j & (G - 1)) * TD_PSTRIDE + (j / G);
-}
-
-// Shared-memory state of one tridiagonalisation of order 8 G.
-template <int G>
-struct TdShared {
-    double up[2][G * TD_PSTRIDE];   // u, permuted (16-byte aligned by the struct's placement)
-    double pp[2][G * TD_PSTRIDE];   // p, permuted
-    double wsum[2][8];
-    double sspart[2][G];            // partial sums of squares of the published row, one per holder thread
-    double dg[8 * G], of[8 * G], ta[8 * G];
-};
-
-// The G threads that hold row r (slot AR = r / G of their tiles) publish its raw tail
-// x = A[r][r+1..] into buffer `nxt`, together with their partial sums of squares of x[r+2..].  The
-// norm, beta and gamma of the reflector are worked out by every thread after the next barrier, in
-// the shadow of the matrix-vector product, instead of by these holders while the CTA waits.
-template <int G, int AR>
-__device__ __forceinline__ void td_publish(const double (&A)[8][8], int r, int nxt, int tc, TdShared<G> &sh) {
-    double x[8];
-    double ss0 = 0.0, ss1 = 0.0;
-#pragma unroll
-    for (int b = 0; b < 8; ++b) {
-        if (b < AR) {
-            x[b] = 0.0;
-        } else {
-            const int j = tc + G * b;
-            const double v = A[AR][b];
-            if (b == AR && j == r) sh.dg[r] = v;
-            x[b] = (j > r) ? v : 0.0;
-            const double t = (j > r + 1) ? v : 0.0;
-            if (b & 1) ss1 = fma(t, t, ss1);
-            else ss0 = fma(t, t, ss0);
-        }
-    }
-    double2 *dst = reinterpret_cast<double2 *>(&sh.up[nxt][tc * TD_PSTRIDE]);
-    dst[0] = make_double2(x[0], x[1]);
-    dst[1] = make_double2(x[2], x[3]);
-    dst[2] = make_double2(x[4], x[5]);
-    dst[3] = make_double2(x[6], x[7]);
-    sh.sspart[nxt][tc] = ss0 + ss1;
-}
-
-// One step k with (k + 1) / G == K0: tile slots below K0 hold only finished rows and columns and
-// are skipped at compile time.  `refl_row` (8 G doubles of shared memory) receives the reflector.
-template <int G, int K0>
-__device__ __forceinline__ void td_step(double (&A)[8][8], int k, int tid, TdShared<G> &sh, double *__restrict__ refl_row) {
-    constexpr int N = 8 * G, NW = G * G / 32;
-    const int lane = tid & 31, warp = tid >> 5, tr = tid / G, tc = tid & (G - 1);
-    __syncthreads();
-    const int cur = k & 1;
-    // reflector scalars from the published row: u = x - beta e_{k+1}, H = I - gamma u u^T
-    double ss;
-    {
-        const double2 *sp = reinterpret_cast<const double2 *>(sh.sspart[cur]);
-        double part[G / 2];
-#pragma unroll
-        for (int q = 0; q < G / 2; ++q) {
-            const double2 v = sp[q];
-            part[q] = v.x + v.y;
-        }
-#pragma unroll
-        for (int w = G / 4; w >= 1; w >>= 1)
-#pragma unroll
-            for (int q = 0; q < w; ++q) part[q] = part[2 * q] + part[2 * q + 1];
-        ss = part[0];
-    }
-    const double alpha = sh.up[cur][td_pos<G>(k + 1)];
-    double beta = alpha, gamma = 0.0;
-    if (ss > 0.0) {
-        const double sq = fma(alpha, alpha, ss);
-        const double nrm = sq * rsqrt(sq);
-        beta = (alpha >= 0.0) ? -nrm : nrm;
-        gamma = 1.0 / fma(fabs(alpha), nrm, sq);   // 1 / (beta (beta - alpha))
-    }
-    if (tid < N) refl_row[tid] = (tid > k) ? sh.up[cur][td_pos<G>(tid)] - ((tid == k + 1) ? beta : 0.0) : 0.0;
-    if (tid == 0) {
-        sh.of[k] = beta;
-        sh.ta[k] = gamma;
-    }
-    const bool owner = (tr == ((k + 1) & (G - 1))) && (k + 1 < N - 2);
-    const bool col_holder = tc == ((k + 1) & (G - 1)), row_holder = tr == ((k + 1) & (G - 1));   // of index k + 1 (tile slot K0)
-    if (gamma != 0.0) {   // uniform over the CTA
-        double uj[8], ui[8], acc[8];
-        {
-            const double2 *src = reinterpret_cast<const double2 *>(&sh.up[cur][tc * TD_PSTRIDE]);
-            const double2 *srow = reinterpret_cast<const double2 *>(&sh.up[cur][tr * TD_PSTRIDE]);
-#pragma unroll
-            for (int q = K0 / 2; q < 4; ++q) {
-                const double2 v = src[q], w = srow[q];
-                uj[2 * q] = v.x;
-                uj[2 * q + 1] = v.y;
-                ui[2 * q] = w.x;
-                ui[2 * q + 1] = w.y;
-            }
-        }
-        // A x with the raw row (independent of beta, so it overlaps the square root and the division
-        // above), then the - beta A e_{k+1} term from the threads that hold column k + 1
-#pragma unroll
-        for (int a = 0; a < 8; ++a) {
-            acc[a] = 0.0;
-            if (a >= K0) {
-                double s0 = 0.0, s1 = 0.0;
-#pragma unroll
-                for (int b = K0; b < 8; ++b) {
-                    if ((b - K0) & 1) s1 = fma(A[a][b], uj[b], s1);
-                    else s0 = fma(A[a][b], uj[b], s0);
-                }
-                acc[a] = s0 + s1;
-            }
-        }
-        double tloc = 0.0;
-        if (col_holder) uj[K0] -= beta;
-        if (row_holder) ui[K0] -= beta;
-#pragma unroll
-        for (int a = K0; a < 8; ++a) {
-            if (col_holder) acc[a] = fma(-beta, A[a][K0], acc[a]);
-            tloc = fma(ui[a], acc[a], tloc);
-        }
-        // sum the partial rows over the G column groups: each stage keeps half of the rows
-        const bool hA = tc & (G / 2), hB = tc & (G / 4), hC = tc & (G / 8);
-        double v4[4], v2[2], v1;
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const double keep = hA ? acc[q + 4] : acc[q], send = hA ? acc[q] : acc[q + 4];
-            v4[q] = keep + __shfl_xor_sync(0xffffffffu, send, G / 2);
-        }
-#pragma unroll
-        for (int q = 0; q < 2; ++q) {
-            const double keep = hB ? v4[q + 2] : v4[q], send = hB ? v4[q] : v4[q + 2];
-            v2[q] = keep + __shfl_xor_sync(0xffffffffu, send, G / 4);
-        }
-        {
-            const double keep = hC ? v2[1] : v2[0], send = hC ? v2[0] : v2[1];
-            v1 = keep + __shfl_xor_sync(0xffffffffu, send, G / 8);
-        }
-        if (G == 16) v1 += __shfl_xor_sync(0xffffffffu, v1, 1);   // two threads per row are left: both get the sum
-        const int arow = (hA ? 4 : 0) + (hB ? 2 : 0) + (hC ? 1 : 0);
-        const int irow = tr + G * arow;
-        if ((G == 8 || !(tc & 1)) && irow > k) sh.pp[cur][td_pos<G>(irow)] = gamma * v1;
-        tloc = warp_sum(tloc);
-        if (lane == 0) sh.wsum[cur][warp] = tloc;
-        __syncthreads();
-        double uAu;
-        {
-            const double2 *wp = reinterpret_cast<const double2 *>(&sh.wsum[cur][0]);
-            const double2 w0 = wp[0];
-            uAu = w0.x + w0.y;
-            if (NW == 8) {
-                const double2 w1 = wp[1], w2 = wp[2], w3 = wp[3];
-                uAu = (uAu + (w1.x + w1.y)) + ((w2.x + w2.y) + (w3.x + w3.y));
-            }
-        }
-        const double twoK = gamma * gamma * uAu;
-        double pj[8], si[8];
-        {
-            const double2 *src = reinterpret_cast<const double2 *>(&sh.pp[cur][tc * TD_PSTRIDE]);
-            const double2 *srow = reinterpret_cast<const double2 *>(&sh.pp[cur][tr * TD_PSTRIDE]);
-#pragma unroll
-            for (int q = K0 / 2; q < 4; ++q) {
-                const double2 v = src[q], w = srow[q];
-                pj[2 * q] = v.x;
-                pj[2 * q + 1] = v.y;
-                si[2 * q] = fma(-twoK, ui[2 * q], w.x);       // p_i - 2 K u_i
-                si[2 * q + 1] = fma(-twoK, ui[2 * q + 1], w.y);
-            }
-        }
-        // The next reflector comes from row k + 1 (slot K0 of its holders): bring that row up to
-        // date and publish it first, so that the other warps' updates hide its latency.
-        if (owner) {
-#pragma unroll
-            for (int b = K0; b < 8; ++b) A[K0][b] = fma(-ui[K0], pj[b], fma(-si[K0], uj[b], A[K0][b]));
-            td_publish<G, K0>(A, k + 1, cur ^ 1, tc, sh);
-        }
-#pragma unroll
-        for (int a = K0; a < 8; ++a) {
-            if (a > K0 || !owner) {
-#pragma unroll
-                for (int b = K0; b < 8; ++b) A[a][b] = fma(-ui[a], pj[b], fma(-si[a], uj[b], A[a][b]));
-            }
-        }
-    } else if (owner) {
-        td_publish<G, K0>(A, k + 1, cur ^ 1, tc, sh);
-    }
-}
-
-template <int G, int K0, int LO, int HI>
-__device__ __forceinline__ void td_step_if(double (&A)[8][8], int k, int tid, TdShared<G> &sh, double *__restrict__ refl_row) {
-    if constexpr (K0 >= LO && K0 <= HI) td_step<G, K0>(A, k, tid, sh, refl_row);
-}
-
-// Steps [KB, KE) of the tridiagonalisation of the order-8G matrix whose element (i, j) sits at
-// gram[(ORIGIN + i) D + ORIGIN + j].  KB and KE are multiples of G, or KE = 8 G - 2 (the last step).
-// The trailing matrix is read from, and when steps remain written back to, its own place in
-// global memory; reflector rows ORIGIN + KB .. ORIGIN + KE - 1 then overwrite rows that are no
-// longer part of it.  Only the tile slots from KB / G up are ever live, so a kernel that starts
-// late needs fewer registers and more of its CTAs fit on an SM.
-template <int G, int ORIGIN, int KB, int KE, int MINB>
-__global__ void __launch_bounds__(G * G, MINB) tridiag_range_kernel(double *__restrict__ gram, double *__restrict__ diag,
-                                                                     double *__restrict__ off, double *__restrict__ tau,
-                                                                     const int *__restrict__ list, const int *__restrict__ count) {
-    constexpr int N = 8 * G, THREADS = G * G, S0 = KB / G;
-    constexpr bool LAST = (KE == N - 2);
-    static_assert(KB % G == 0 && (LAST || KE % G == 0), "ranges start and end on tile-slot boundaries");
-    __shared__ __align__(16) double refl[(KE - KB) * N];   // the reflectors of this range
-    __shared__ __align__(16) TdShared<G> sh;
-    const int tid = threadIdx.x;
-    const int tr = tid / G, tc = tid & (G - 1);
-    // without a list: block blockIdx.x; with one: the listed blocks, shared out over the grid
-    for (int li = blockIdx.x; !list || li < *count; li += gridDim.x) {
-    const int blk = list ? list[li] : li;
-    double *Gm = gram + static_cast<size_t>(blk) * D * D;
-    double *T = Gm + static_cast<size_t>(ORIGIN) * D + ORIGIN;
-
-    double A[8][8];
-#pragma unroll
-    for (int a = S0; a < 8; ++a)
-#pragma unroll
-        for (int b = S0; b < 8; ++b) A[a][b] = T[static_cast<size_t>(tr + G * a) * D + tc + G * b];
-    for (int e = tid; e < G * TD_PSTRIDE; e += THREADS) {
-        sh.up[0][e] = 0.0;
-        sh.up[1][e] = 0.0;
-        sh.pp[0][e] = 0.0;
-        sh.pp[1][e] = 0.0;
-    }
-    __syncthreads();
-
-    if (tr == 0) td_publish<G, S0>(A, KB, KB & 1, tc, sh);
-    constexpr int LO = (KB + 1) / G, HI = (LAST ? KE - 1 : KE) / G;
-#pragma unroll 1
-    for (int k = KB; k < KE; ++k) {
-        double *row = refl + (k - KB) * N;
-        switch ((k + 1) / G) {
-            case 0: td_step_if<G, 0, LO, HI>(A, k, tid, sh, row); break;
-            case 1: td_step_if<G, 1, LO, HI>(A, k, tid, sh, row); break;
-            case 2: td_step_if<G, 2, LO, HI>(A, k, tid, sh, row); break;
-            case 3: td_step_if<G, 3, LO, HI>(A, k, tid, sh, row); break;
-            case 4: td_step_if<G, 4, LO, HI>(A, k, tid, sh, row); break;
-            case 5: td_step_if<G, 5, LO, HI>(A, k, tid, sh, row); break;
-            case 6: td_step_if<G, 6, LO, HI>(A, k, tid, sh, row); break;
-            default: td_step_if<G, 7, LO, HI>(A, k, tid, sh, row); break;
-        }
-    }
-    if (LAST) {
-        if (tid == (G - 2) * G + G - 2) sh.dg[N - 2] = A[7][7];
-        if (tid == (G - 2) * G + G - 1) sh.of[N - 2] = A[7][7];
-        if (tid == (G - 1) * G + G - 1) sh.dg[N - 1] = A[7][7];
-        if (tid == 0) {
-            sh.of[N - 1] = 0.0;
-            sh.ta[N - 2] = 0.0;
-            sh.ta[N - 1] = 0.0;
-        }
-    }
-    __syncthreads();
-    // reflector of step k: zero up to column ORIGIN + k, in the full-width row ORIGIN + k
-    for (int e = tid; e < (KE - KB) * (D / 2); e += THREADS) {
-        const int r = e / (D / 2), c2 = e % (D / 2);
-        const double2 v = (c2 < ORIGIN / 2) ? make_double2(0.0, 0.0) : reinterpret_cast<const double2 *>(refl + r * N)[c2 - ORIGIN / 2];
-        reinterpret_cast<double2 *>(Gm + static_cast<size_t>(ORIGIN + KB + r) * D)[c2] = v;
-    }
-    if (!LAST) {
-        constexpr int S1 = KE / G;
-#pragma unroll
-        for (int a = S1; a < 8; ++a)
-#pragma unroll
-            for (int b = S1; b < 8; ++b) T[static_cast<size_t>(tr + G * a) * D + tc + G * b] = A[a][b];
-    }
-    constexpr int KOUT = LAST ? N : KE;
-    for (int k = KB + tid; k < KOUT; k += THREADS) {
-        const size_t o = static_cast<size_t>(blk) * D + ORIGIN + k;
-        diag[o] = sh.dg[k];
-        off[o] = sh.of[k];
-        tau[o] = sh.ta[k];
-    }
-    if (!list) break;
-    __syncthreads();   // the shared state is reused by the next listed block
-    }
-}
-
-// ------------------------------------------------------------------------------------------
 // Eigenvalues of a symmetric tridiagonal matrix from Sturm sequences: with
 //   p_0 = 1, p_1 = d_0 - x, p_{i+1} = (d_i - x) p_i - e_{i-1}^2 p_{i-1},
 // the number of sign changes in p_0 .. p_d is the number of eigenvalues below x, and p_d(x) is the
@@ -927,18 +624,6 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
         ws.rank[b] = rank;
         out.status[gb] = static_cast<int32_t>(s_flags);
         if (out.lambda_plus) out.lambda_plus[gb] = static_cast<float>(lam_plus);
-    }
-}
-
-// The three ranges: order 128 with one CTA per SM while every tile slot is live, two CTAs per SM
-// from step 32, and the trailing 64 x 64 matrix on 64 threads with four CTAs per SM.
-void launch_tridiag(int part, int64_t nb, const Workspace &ws, const int *list, const int *count, cudaStream_t s) {
-    const unsigned g = list_grid(nb, list);
-    double *g0 = ws.gram, *d0 = ws.diag, *o0 = ws.off, *t0 = ws.tau;
-    switch (part) {
-        case 0: tridiag_range_kernel<16, 0, 0, 32, 1><<<g, 256, 0, s>>>(g0, d0, o0, t0, list, count); break;
-        case 1: tridiag_range_kernel<16, 0, 32, 64, 2><<<g, 256, 0, s>>>(g0, d0, o0, t0, list, count); break;
-        default: tridiag_range_kernel<8, 64, 0, 62, 4><<<g, 64, 0, s>>>(g0, d0, o0, t0, list, count); break;
     }
 }
 

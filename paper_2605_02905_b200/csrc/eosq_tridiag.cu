@@ -1,0 +1,469 @@
+// Householder tridiagonalisation of the d x d Gram matrices (the first half of the symmetric
+// eigen-decomposition that stands in for the block's SVD, Sec. 2.3 and Algorithm 2 REQUIRE line),
+// in double precision, with the matrix resident in tensor memory.
+//
+// Why tensor memory.  Every step of the reduction is a chain of dependent latencies (publish a row,
+// barrier, norm, matrix-vector product, reduction, barrier, rank-2 update), so one matrix cannot
+// keep the double-precision pipe of an SM busy: several matrices per SM have to be in flight, each
+// worked on by enough warps to keep its own steps short.  A 128 x 128 fp64 matrix is 128 KB, half
+// of the register file, so registers hold one.  Tensor memory (256 KB per SM, 128 lanes x 512
+// columns of 32 bits) is otherwise idle here and is addressed per thread: a thread of warp w reads
+// and writes lane 32 (w % 4) + its lane index, any columns, with tcgen05.ld / tcgen05.st.  With the
+// matrix there, a thread needs registers only for the vectors of a step, 128 registers are enough,
+// and sixteen warps fit on an SM: two matrices of order 128 (256 threads each), or eight of order
+// 64 (64 threads each).
+//
+// Layout.  A team of G x G threads (G = order / 8) works on one matrix; thread (tr, tc) =
+// (t / G, t % G) holds A[tr + G a][tc + G b], a, b < 8, so every thread keeps an equal share of the
+// shrinking trailing matrix.  Row slot a of a thread's tile is 16 consecutive tensor-memory columns
+// (eight doubles), one load or store instruction.
+//
+// One step k reflects with H = I - gamma u u^T, u = x - beta e_{k+1}, x = A[k][k+1..],
+// beta = -sign(x_{k+1}) ||x||, gamma = 1 / (beta (beta - x_{k+1})):
+//     p = gamma A u,  2K = gamma (u . p),  A <- A - u p^T - (p - 2K u) u^T.
+// The rank-2 update of step k is not applied when it becomes known but folded into the sweep of
+// step k + 1, which reads every live element once, brings it up to date, writes it back and uses it
+// for the next matrix-vector product: one pass over tensor memory per step instead of two.  Only
+// the row that defines the next reflector is brought up to date early, by the G threads that hold
+// it.  x and p travel through shared memory (double buffered by the parity of k, two team-wide
+// barriers per step) in a permuted order that makes a thread's eight columns contiguous.
+// Finished tile slots are skipped at compile time (one instantiation of the step per value of
+// (k + 1) / G).
+#include <algorithm>
+
+#include "eosq_common.cuh"
+#include "eosq_sm100.cuh"
+
+namespace eosq {
+
+using namespace sm100;
+
+namespace {
+
+constexpr int TT_PSTRIDE = 10;   // doubles per column residue in the permuted vectors (8 used, 2 pad)
+
+// 16 columns of the thread's lane; the wait carries the registers, so that no use of them can be
+// scheduled ahead of it.
+__device__ __forceinline__ void tt_wait16(uint32_t (&r)[16]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
+                   "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
+                 :
+                 : "memory");
+}
+__device__ __forceinline__ void tt_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+        :
+        : "r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
+__device__ __forceinline__ double tt_get(const uint32_t (&r)[16], int e) {
+    return __hiloint2double(static_cast<int>(r[2 * e + 1]), static_cast<int>(r[2 * e]));
+}
+__device__ __forceinline__ void tt_put(uint32_t (&r)[16], int e, double v) {
+    r[2 * e] = static_cast<uint32_t>(__double2loint(v));
+    r[2 * e + 1] = static_cast<uint32_t>(__double2hiint(v));
+}
+// Barrier over the threads of one team (the whole CTA when it is one team).
+template <int TEAMS, int TEAM_THREADS>
+__device__ __forceinline__ void tt_sync(int team) {
+    // the barrier number is spelled out: a number in a register makes the compiler reserve all sixteen
+    // barriers for the CTA, and the SM then holds two CTAs instead of four
+    if (TEAMS == 1) __syncthreads();
+    else if (team == 0) asm volatile("bar.sync 1, %0;" ::"n"(TEAM_THREADS) : "memory");
+    else if (team == 1) asm volatile("bar.sync 2, %0;" ::"n"(TEAM_THREADS) : "memory");
+    else if (team == 2) asm volatile("bar.sync 3, %0;" ::"n"(TEAM_THREADS) : "memory");
+    else asm volatile("bar.sync 4, %0;" ::"n"(TEAM_THREADS) : "memory");
+}
+// 1 / sqrt(x) and 1 / x to a few ulp: the hardware's estimates (about 2^-22) and two Newton steps.
+// Both sit on the chain that every step waits for; x is a sum of squares well inside the normal range
+// (a subnormal or huge x only costs accuracy on a matrix whose scale is already hopeless).
+__device__ __forceinline__ double tt_rsqrt(double x) {
+    double y;
+    asm("rsqrt.approx.ftz.f64 %0, %1;" : "=d"(y) : "d"(x));
+    const double hx = 0.5 * x;
+    double e = fma(-hx * y, y, 0.5);
+    y = fma(y, e, y);
+    e = fma(-hx * y, y, 0.5);
+    return fma(y, e, y);
+}
+__device__ __forceinline__ double tt_rcp(double x) {
+    double r;
+    asm("rcp.approx.ftz.f64 %0, %1;" : "=d"(r) : "d"(x));
+    double e = fma(-x, r, 1.0);
+    r = fma(r, e, r);
+    e = fma(-x, r, 1.0);
+    return fma(r, e, r);
+}
+template <int G>
+__device__ __forceinline__ int tt_pos(int j) {
+    return (j & (G - 1)) * TT_PSTRIDE + (j / G);
+}
+
+// Shared-memory state of one reduction of order 8 G.
+template <int G>
+struct TtShared {
+    double xu[2][G * TT_PSTRIDE];   // published row x (zero up to its own index), permuted
+    double pp[2][G * TT_PSTRIDE];   // p, permuted (zero for finished indices)
+    double sspart[2][G];            // partial sums of squares of x[k+2..], one per publishing thread
+    double wsum[2][8];              // per-warp parts of u . A u
+    double dg[8 * G], of[8 * G], ta[8 * G];
+};
+
+// The G threads that hold row r (row slot AR = r / G of their tiles) publish x = A[r][r+1..] into
+// buffer `nxt`.  With UPDATE the pending rank-2 update of step r - 1 (vectors in buffer nxt ^ 1,
+// u_{r-1}[r] = uown, (p - 2K u)[r] = sown) is applied to the row first; the stored row is left as
+// it is, the next sweep brings it up to date like every other row.  Tensor-memory loads are
+// warp-wide instructions, so the whole warp of the holders runs this and `mine` marks the holders.
+template <int G, int AR, bool UPDATE>
+__device__ __forceinline__ void tt_publish(uint32_t tb, int r, int nxt, int tc, bool mine, TtShared<G> &sh, double uown, double sown) {
+    uint32_t raw[16];
+    tmem_ld16(tb + 16u * AR, raw);
+    double uj[8], pj[8];
+    if (UPDATE) {
+        const double2 *us = reinterpret_cast<const double2 *>(&sh.xu[nxt ^ 1][tc * TT_PSTRIDE]);
+        const double2 *ps = reinterpret_cast<const double2 *>(&sh.pp[nxt ^ 1][tc * TT_PSTRIDE]);
+#pragma unroll
+        for (int q = AR / 2; q < 4; ++q) {
+            const double2 v = us[q], w = ps[q];
+            uj[2 * q] = v.x;
+            uj[2 * q + 1] = v.y;
+            pj[2 * q] = w.x;
+            pj[2 * q + 1] = w.y;
+        }
+    }
+    tt_wait16(raw);
+    double x[8], ss0 = 0.0, ss1 = 0.0;
+#pragma unroll
+    for (int b = 0; b < 8; ++b) {
+        if (b < AR) {
+            x[b] = 0.0;
+            continue;
+        }
+        const int col = tc + G * b;
+        double t = tt_get(raw, b);
+        if (UPDATE) {
+            // u_{r-1} at index r is x - beta, which is uown; right of it the raw x is u
+            const double ujf = (b == AR && col == r) ? uown : uj[b];
+            t = fma(-uown, pj[b], fma(-sown, ujf, t));
+        }
+        if (b == AR && mine && col == r) sh.dg[r] = t;
+        x[b] = (col > r) ? t : 0.0;
+        const double s = (col > r + 1) ? t : 0.0;
+        if (b & 1) ss1 = fma(s, s, ss1);
+        else ss0 = fma(s, s, ss0);
+    }
+    if (mine) {
+        double2 *dst = reinterpret_cast<double2 *>(&sh.xu[nxt][tc * TT_PSTRIDE]);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) dst[q] = make_double2(x[2 * q], x[2 * q + 1]);
+        sh.sspart[nxt][tc] = ss0 + ss1;
+    }
+}
+
+// One step k of a team, with (k + 1) / G == K0.  `grow` is the global row that receives the
+// reflector; t is the thread's index within its team.  twoK of the pending update comes in, that
+// of this step goes out.
+template <int G, int K0, int TEAMS>
+__device__ __forceinline__ void tt_step(uint32_t tb, int k, int kend, int t, int team, TtShared<G> &sh, double *__restrict__ grow,
+                                        double &twoK_prev) {
+    constexpr int N = 8 * G, TEAM_THREADS = G * G, NW = TEAM_THREADS / 32;
+    const int lane = t & 31, warp = t >> 5, tr = t / G, tc = t & (G - 1);
+    tt_sync<TEAMS, TEAM_THREADS>(team);
+    const int cur = k & 1, prv = cur ^ 1;
+    // reflector scalars from the published row
+    double ss;
+    {
+        const double2 *sp = reinterpret_cast<const double2 *>(sh.sspart[cur]);
+        double part[G / 2];
+#pragma unroll
+        for (int q = 0; q < G / 2; ++q) {
+            const double2 v = sp[q];
+            part[q] = v.x + v.y;
+        }
+#pragma unroll
+        for (int w = G / 4; w >= 1; w >>= 1)
+#pragma unroll
+            for (int q = 0; q < w; ++q) part[q] = part[2 * q] + part[2 * q + 1];
+        ss = part[0];
+    }
+    const double alpha = sh.xu[cur][tt_pos<G>(k + 1)];
+    double beta = alpha, gamma = 0.0;
+    if (ss > 0.0) {
+        const double sq = fma(alpha, alpha, ss);
+        const double nrm = sq * tt_rsqrt(sq);
+        beta = (alpha >= 0.0) ? -nrm : nrm;
+        gamma = tt_rcp(fma(fabs(alpha), nrm, sq));   // 1 / (beta (beta - alpha))
+    }
+    if (t < N) grow[t] = (t > k) ? sh.xu[cur][tt_pos<G>(t)] - ((t == k + 1) ? beta : 0.0) : 0.0;
+    if (t == 0) {
+        sh.of[k] = beta;
+        sh.ta[k] = gamma;
+    }
+    const bool col_holder = tc == ((k + 1) & (G - 1)), row_holder = tr == ((k + 1) & (G - 1));   // of index k + 1 (slot K0)
+    // column-side vectors: u of this step, u' and p' of the pending update
+    double ujn[8], ujp[8], pjp[8];
+    {
+        const double2 *un = reinterpret_cast<const double2 *>(&sh.xu[cur][tc * TT_PSTRIDE]);
+        const double2 *up = reinterpret_cast<const double2 *>(&sh.xu[prv][tc * TT_PSTRIDE]);
+        const double2 *pq = reinterpret_cast<const double2 *>(&sh.pp[prv][tc * TT_PSTRIDE]);
+#pragma unroll
+        for (int q = K0 / 2; q < 4; ++q) {
+            const double2 a = un[q], b = up[q], c = pq[q];
+            ujn[2 * q] = a.x;
+            ujn[2 * q + 1] = a.y;
+            ujp[2 * q] = b.x;
+            ujp[2 * q + 1] = b.y;
+            pjp[2 * q] = c.x;
+            pjp[2 * q + 1] = c.y;
+        }
+        if (col_holder) ujn[K0] -= beta;
+    }
+    // The sweep: every live element is brought up to date, written back and used for A u.  The
+    // pending update needs no correction at index k (u' there is x' - beta'): row and column k are
+    // finished and nothing reads them again.
+    double acc[8];
+    const double *ur = &sh.xu[prv][tr * TT_PSTRIDE], *pr = &sh.pp[prv][tr * TT_PSTRIDE];
+#pragma unroll
+    for (int a = 0; a < 8; ++a) {
+        acc[a] = 0.0;
+        if (a < K0) continue;
+        uint32_t raw[16];
+        tmem_ld16(tb + 16u * a, raw);
+        const double uip = ur[a];
+        const double sip = fma(-twoK_prev, uip, pr[a]);
+        tt_wait16(raw);
+        double s0 = 0.0, s1 = 0.0;
+#pragma unroll
+        for (int b = K0; b < 8; ++b) {
+            double v = tt_get(raw, b);
+            v = fma(-uip, pjp[b], v);
+            v = fma(-sip, ujp[b], v);
+            tt_put(raw, b, v);
+            if ((b - K0) & 1) s1 = fma(v, ujn[b], s1);
+            else s0 = fma(v, ujn[b], s0);
+        }
+        tt_st16(tb + 16u * a, raw);
+        acc[a] = s0 + s1;
+    }
+    // u . A u (parts), then the sums of the partial rows over the G column residues: each stage
+    // keeps half of the rows
+    double tloc = 0.0;
+    {
+        const double2 *un = reinterpret_cast<const double2 *>(&sh.xu[cur][tr * TT_PSTRIDE]);
+        double uin[8];
+#pragma unroll
+        for (int q = K0 / 2; q < 4; ++q) {
+            const double2 v = un[q];
+            uin[2 * q] = v.x;
+            uin[2 * q + 1] = v.y;
+        }
+        if (row_holder) uin[K0] -= beta;
+#pragma unroll
+        for (int a = K0; a < 8; ++a) tloc = fma(uin[a], acc[a], tloc);
+    }
+    const bool hA = tc & (G / 2), hB = tc & (G / 4), hC = tc & (G / 8);
+    double v4[4], v2[2], v1;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const double keep = hA ? acc[q + 4] : acc[q], send = hA ? acc[q] : acc[q + 4];
+        v4[q] = keep + __shfl_xor_sync(0xffffffffu, send, G / 2);
+    }
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+        const double keep = hB ? v4[q + 2] : v4[q], send = hB ? v4[q] : v4[q + 2];
+        v2[q] = keep + __shfl_xor_sync(0xffffffffu, send, G / 4);
+    }
+    {
+        const double keep = hC ? v2[1] : v2[0], send = hC ? v2[0] : v2[1];
+        v1 = keep + __shfl_xor_sync(0xffffffffu, send, G / 8);
+    }
+    if (G == 16) v1 += __shfl_xor_sync(0xffffffffu, v1, 1);   // two threads per row are left: both get the sum
+    const int arow = (hA ? 4 : 0) + (hB ? 2 : 0) + (hC ? 1 : 0);
+    const int irow = tr + G * arow;
+    if (G == 8 || !(tc & 1)) sh.pp[cur][tt_pos<G>(irow)] = (irow > k) ? gamma * v1 : 0.0;
+    tloc = warp_sum(tloc);
+    if (lane == 0) sh.wsum[cur][warp] = tloc;
+    tmem_st_wait();   // this thread's own stores; nobody else reads its lane
+    tt_sync<TEAMS, TEAM_THREADS>(team);
+    double uAu;
+    {
+        const double2 *wp = reinterpret_cast<const double2 *>(&sh.wsum[cur][0]);
+        const double2 w0 = wp[0];
+        uAu = w0.x + w0.y;
+        if (NW == 8) {
+            const double2 w1 = wp[1], w2 = wp[2], w3 = wp[3];
+            uAu = (uAu + (w1.x + w1.y)) + ((w2.x + w2.y) + (w3.x + w3.y));
+        }
+    }
+    const double twoK = gamma * gamma * uAu;
+    twoK_prev = twoK;
+    // the next reflector comes from row k + 1 (row slot K0 of its G holders, all in one warp)
+    if (k + 1 < kend && warp == (((k + 1) & (G - 1)) * G) / 32) {
+        const int p1 = tt_pos<G>(k + 1);
+        const double uown = sh.xu[cur][p1] - beta;
+        const double sown = fma(-twoK, uown, sh.pp[cur][p1]);
+        tt_publish<G, K0, true>(tb, k + 1, prv, tc, row_holder, sh, uown, sown);
+    }
+}
+
+template <int G, int K0, int LO, int HI, int TEAMS>
+__device__ __forceinline__ void tt_step_if(uint32_t tb, int k, int kend, int t, int team, TtShared<G> &sh, double *__restrict__ grow,
+                                           double &twoK_prev) {
+    if constexpr (K0 >= LO && K0 <= HI) tt_step<G, K0, TEAMS>(tb, k, kend, t, team, sh, grow, twoK_prev);
+}
+
+// Steps [0, KE) of the reduction of the order-8G matrix whose element (i, j) sits at
+// gram[(ORIGIN + i) D + ORIGIN + j]; KE is a multiple of G, or 8 G - 2 (the last step).  Reflector
+// k goes to row ORIGIN + k (full width, zero up to column ORIGIN + k); diag / off / tau receive
+// d_k, the new off-diagonal entry and gamma_k.  When steps remain the trailing matrix is written
+// back to its own place.  A CTA holds TEAMS teams, each working through its own matrices.
+template <int G, int ORIGIN, int KE, int TEAMS, int MINB>
+__global__ void __launch_bounds__(G *G *TEAMS, MINB) tridiag_tm_kernel(double *__restrict__ gram, double *__restrict__ diag,
+                                                                        double *__restrict__ off, double *__restrict__ tau, int nb,
+                                                                        const int *__restrict__ list, const int *__restrict__ count) {
+    constexpr int N = 8 * G, TEAM_THREADS = G * G, THREADS = TEAM_THREADS * TEAMS;
+    // columns per CTA: a thread's tile is 128 columns, and warps w, w + 4 share the lanes of a quadrant
+    constexpr uint32_t COLS = 128u * ((THREADS / 32 + 3) / 4);
+    constexpr bool LAST = (KE == N - 2);
+    static_assert(LAST || KE % G == 0, "ranges end on tile-slot boundaries");
+    static_assert(COLS >= 32 && (COLS & (COLS - 1)) == 0 && COLS <= 512, "tensor-memory allocations are powers of two");
+    static_assert(TEAM_THREADS % 32 == 0, "teams are whole warps");
+    __shared__ __align__(16) TtShared<G> shs[TEAMS];
+    __shared__ uint32_t tmem_base_s;
+    const int tid = threadIdx.x, cwarp = tid >> 5;
+    const int team = tid / TEAM_THREADS, t = tid % TEAM_THREADS;
+    const int tr = t / G, tc = t & (G - 1);
+    TtShared<G> &sh = shs[team];
+    if (cwarp == 0) {
+        tmem_alloc(&tmem_base_s, COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tb = tmem_base_s + (static_cast<uint32_t>(32 * (cwarp & 3)) << 16) + 128u * static_cast<uint32_t>(cwarp >> 2);
+    const int total = list ? *count : nb;
+    for (int li = blockIdx.x * TEAMS + team; li < total; li += gridDim.x * TEAMS) {
+        const int blk = list ? list[li] : li;
+        double *Gm = gram + static_cast<size_t>(blk) * D * D;
+        double *T = Gm + static_cast<size_t>(ORIGIN) * D + ORIGIN;
+        // the matrix into tensor memory
+#pragma unroll
+        for (int a = 0; a < 8; ++a) {
+            uint32_t raw[16];
+#pragma unroll
+            for (int b = 0; b < 8; ++b) tt_put(raw, b, T[static_cast<size_t>(tr + G * a) * D + tc + G * b]);
+            tt_st16(tb + 16u * a, raw);
+        }
+        for (int e = t; e < G * TT_PSTRIDE; e += TEAM_THREADS) {
+            sh.xu[0][e] = 0.0;
+            sh.xu[1][e] = 0.0;
+            sh.pp[0][e] = 0.0;
+            sh.pp[1][e] = 0.0;
+        }
+        if constexpr (ORIGIN > 0) {   // the reflector rows of this range are full-width rows: zero left of the matrix
+            for (int e = t; e < KE * (ORIGIN / 2); e += TEAM_THREADS) {
+                const int r = e / (ORIGIN / 2), c2 = e % (ORIGIN / 2);
+                reinterpret_cast<double2 *>(Gm + static_cast<size_t>(ORIGIN + r) * D)[c2] = make_double2(0.0, 0.0);
+            }
+        }
+        tmem_st_wait();
+        tt_sync<TEAMS, TEAM_THREADS>(team);
+        if ((t >> 5) == 0) tt_publish<G, 0, false>(tb, 0, 0, tc, tr == 0, sh, 0.0, 0.0);
+        double twoK_prev = 0.0;
+        constexpr int HI = KE / G;
+#pragma unroll 1
+        for (int k = 0; k < KE; ++k) {
+            double *grow = Gm + static_cast<size_t>(ORIGIN + k) * D + ORIGIN;
+            switch ((k + 1) / G) {
+                case 0: tt_step_if<G, 0, 0, HI, TEAMS>(tb, k, KE, t, team, sh, grow, twoK_prev); break;
+                case 1: tt_step_if<G, 1, 0, HI, TEAMS>(tb, k, KE, t, team, sh, grow, twoK_prev); break;
+                case 2: tt_step_if<G, 2, 0, HI, TEAMS>(tb, k, KE, t, team, sh, grow, twoK_prev); break;
+                case 3: tt_step_if<G, 3, 0, HI, TEAMS>(tb, k, KE, t, team, sh, grow, twoK_prev); break;
+                case 4: tt_step_if<G, 4, 0, HI, TEAMS>(tb, k, KE, t, team, sh, grow, twoK_prev); break;
+                case 5: tt_step_if<G, 5, 0, HI, TEAMS>(tb, k, KE, t, team, sh, grow, twoK_prev); break;
+                case 6: tt_step_if<G, 6, 0, HI, TEAMS>(tb, k, KE, t, team, sh, grow, twoK_prev); break;
+                default: tt_step_if<G, 7, 0, HI, TEAMS>(tb, k, KE, t, team, sh, grow, twoK_prev); break;
+            }
+        }
+        // The update of the last step is still pending: apply it to what is left of the matrix
+        // (rows and columns from KE on) and hand that on: to global memory for the next kernel, or,
+        // at the very end, as the last diagonal and off-diagonal entries.
+        {
+            constexpr int AF = KE / G;
+            const int kl = KE - 1, cur = kl & 1;
+            const double beta = sh.of[kl];
+            double uj[8], pj[8];
+#pragma unroll
+            for (int b = AF; b < 8; ++b) {
+                const int col = tc + G * b;
+                uj[b] = sh.xu[cur][tc * TT_PSTRIDE + b] - ((col == KE) ? beta : 0.0);
+                pj[b] = sh.pp[cur][tc * TT_PSTRIDE + b];
+            }
+#pragma unroll
+            for (int a = AF; a < 8; ++a) {
+                const int row = tr + G * a;
+                const double ui = sh.xu[cur][tr * TT_PSTRIDE + a] - ((row == KE) ? beta : 0.0);
+                const double si = fma(-twoK_prev, ui, sh.pp[cur][tr * TT_PSTRIDE + a]);
+                uint32_t raw[16];
+                tmem_ld16(tb + 16u * a, raw);
+                tt_wait16(raw);
+#pragma unroll
+                for (int b = AF; b < 8; ++b) {
+                    const int col = tc + G * b;
+                    const double v = fma(-ui, pj[b], fma(-si, uj[b], tt_get(raw, b)));
+                    if (LAST) {
+                        if (row == N - 2 && col == N - 2) sh.dg[N - 2] = v;
+                        if (row == N - 2 && col == N - 1) sh.of[N - 2] = v;
+                        if (row == N - 1 && col == N - 1) sh.dg[N - 1] = v;
+                    } else if (row >= KE && col >= KE) {
+                        T[static_cast<size_t>(row) * D + col] = v;
+                    }
+                }
+            }
+            if (LAST && t == 0) {
+                sh.of[N - 1] = 0.0;
+                sh.ta[N - 2] = 0.0;
+                sh.ta[N - 1] = 0.0;
+            }
+        }
+        tt_sync<TEAMS, TEAM_THREADS>(team);
+        constexpr int KOUT = LAST ? N : KE;
+        for (int k = t; k < KOUT; k += TEAM_THREADS) {
+            const size_t o = static_cast<size_t>(blk) * D + ORIGIN + k;
+            diag[o] = sh.dg[k];
+            off[o] = sh.of[k];
+            tau[o] = sh.ta[k];
+        }
+        tt_sync<TEAMS, TEAM_THREADS>(team);   // the shared state is reused by the team's next block
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (cwarp == 0) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base_s, COLS);
+    }
+}
+
+}  // namespace
+
+// Two ranges: the 128 x 128 matrix through its first 64 steps (256 threads and 256 columns of
+// tensor memory per matrix, two CTAs per SM), then the trailing 64 x 64 matrix (teams of 64
+// threads, two per CTA, four CTAs per SM).
+void launch_tridiag(int part, int64_t nb, const Workspace &ws, const int *list, const int *count, int sm_count, cudaStream_t s) {
+    double *g0 = ws.gram, *d0 = ws.diag, *o0 = ws.off, *t0 = ws.tau;
+    const int n = static_cast<int>(nb);
+    const int64_t work = list ? std::min<int64_t>(nb, LIST_GRID) : nb;
+    if (part == 0) {
+        const int grid = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(work, 2 * static_cast<int64_t>(sm_count))));
+        tridiag_tm_kernel<16, 0, 64, 1, 2><<<grid, 256, 0, s>>>(g0, d0, o0, t0, n, list, count);
+    } else {
+        const int grid = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>((work + 1) / 2, 4 * static_cast<int64_t>(sm_count))));
+        tridiag_tm_kernel<8, 64, 62, 2, 4><<<grid, 128, 0, s>>>(g0, d0, o0, t0, n, list, count);
+    }
+}
+
+}  // namespace eosq
