@@ -222,8 +222,11 @@ class Cache:
             V=torch.empty((B, EOSQ_RMAX, d), dtype=torch.float16, **kw),
             status=torch.empty((B,), dtype=torch.int32, **kw),
         )
-        if diagnostics:
+        # diagnostics: True = every optional array; "staged" = all but the full spectrum `eig`
+        # (asking for `eig` makes eosq_encode resolve all d eigenvalues instead of the 3k + 2 it needs)
+        if diagnostics and diagnostics != "staged":
             c.eig = torch.empty((B, d), dtype=torch.float32, **kw)
+        if diagnostics:
             c.lambda_plus = torch.empty((B,), dtype=torch.float32, **kw)
             c.vr32 = torch.empty((B, EOSQ_RMAX, d), dtype=torch.float32, **kw)
             c.coef = torch.empty((B, EOSQ_RMAX), dtype=torch.float32, **kw)

@@ -133,19 +133,20 @@ int eosq::encode_chunk(eosq_ctx *ctx, const void *blocks, int in_dtype, int64_t 
     } else {
         run_stage(ctx, ST_GRAM, s, [&] { launch_gram_plain(chunk_in, in_dtype, nb, n, ws.gram, nullptr, nullptr, s); });
     }
+    const bool full = out_all.eig != nullptr;   // the optional eigenvalue output asks for the whole spectrum
     static_assert(TRIDIAG_PARTS == 2, "one profiling stage per tridiagonalisation kernel");
     for (int part = 0; part < TRIDIAG_PARTS; ++part)
         run_stage(ctx, ST_TRIDIAG_A + part, s, [&] { launch_tridiag(part, nb, ws, nullptr, nullptr, ctx->sm_count, s); });
     // the eigenvalue kernel also queues, in ws.redo_list, the blocks the tensor-core Gram matrix cannot resolve
-    run_stage(ctx, ST_EIGVALS, s, [&] { launch_eigvals(nb, ws, nullptr, nullptr, (in_dtype == EOSQ_F16) ? ws.redo_list : nullptr, s); });
+    run_stage(ctx, ST_EIGVALS, s, [&] { launch_eigvals(nb, ws, nullptr, nullptr, (in_dtype == EOSQ_F16) ? ws.redo_list : nullptr, full, s); });
     if (in_dtype == EOSQ_F16) {
         // second pass, exact Gram matrix, for those blocks (the spectral kernel clears the queue afterwards)
         run_stage(ctx, ST_REDO, s, [&] { launch_gram_plain(chunk_in, in_dtype, nb, n, ws.gram, ws.redo_list, ws.redo_count, s); });
         for (int part = 0; part < TRIDIAG_PARTS; ++part)
             run_stage(ctx, ST_REDO, s, [&] { launch_tridiag(part, nb, ws, ws.redo_list, ws.redo_count, ctx->sm_count, s); });
-        run_stage(ctx, ST_REDO, s, [&] { launch_eigvals(nb, ws, ws.redo_list, ws.redo_count, nullptr, s); });
+        run_stage(ctx, ST_REDO, s, [&] { launch_eigvals(nb, ws, ws.redo_list, ws.redo_count, nullptr, full, s); });
     }
-    run_stage(ctx, ST_SPECTRAL, s, [&] { launch_spectral(nb, n, ws, o, 0, s); });
+    run_stage(ctx, ST_SPECTRAL, s, [&] { launch_spectral(nb, n, ws, o, 0, full, s); });
     if (in_dtype == EOSQ_F16) {
         bool setup_ok = true;
         run_stage(ctx, ST_QUANT, s, [&] { setup_ok = launch_quant_tc(blocks, b0, nb, n, ws, rot, cb, o, ctx->dev_err, ctx->sm_count, s); });

@@ -134,10 +134,12 @@ inline unsigned list_grid(int64_t nb, const int *list) {
 constexpr int TRIDIAG_PARTS = 2;
 void launch_tridiag(int part, int64_t nb, const Workspace &ws, const int *list, const int *count, int sm_count, cudaStream_t s);
 // All eigenvalues of each tridiagonal matrix by Sturm bisection.
-void launch_eigvals(int64_t nb, const Workspace &ws, const int *list, const int *count, int *mark_list, cudaStream_t s);
+// With `full` every eigenvalue is resolved, otherwise the 3k + 1 largest and the smallest (what
+// Algorithm 2 reads one by one and what the accuracy check of the Gram matrix needs).
+void launch_eigvals(int64_t nb, const Workspace &ws, const int *list, const int *count, int *mark_list, bool full, cudaStream_t s);
 // Clears the redo list / appends every block whose eigenvalue range exceeds 1 / REDO_RATIO.
 // Bulk edge, rank, imputed spectrum, D-transform and shrinkage; kept eigenvectors.
-void launch_spectral(int64_t nb, int n, const Workspace &ws, const eosq_cache_t &out, int64_t block0,
+void launch_spectral(int64_t nb, int n, const Workspace &ws, const eosq_cache_t &out, int64_t block0, bool full,
                      cudaStream_t s);
 // Residual, norm, rotation, codes, packing and left factors.
 void launch_quant_plain(const void *blocks, int in_dtype, int64_t nb, int n, const Workspace &ws,

@@ -82,12 +82,23 @@ __device__ __forceinline__ int sturm_eval(const double2 *__restrict__ sde, doubl
     return static_cast<int>(cnt);
 }
 
+// Which eigenvalues a call resolves.  Algorithm 2 reads individually only lambda_1 .. lambda_{2k+r+1}
+// (Steps 1 and 2; r <= k, so 3k + 1 = 34 of them at d = 128); the rest of the spectrum enters
+// through sums that the spectral kernel takes from the characteristic polynomial.  The smallest
+// eigenvalue is resolved as well: it decides whether the tensor-core Gram matrix was accurate
+// enough.  With FULL every eigenvalue is resolved (the optional `eig` output).
+constexpr int EV_TOP = 3 * KPILOT + 1;
+
 // With `mark_list` set (first pass over tensor-core Gram matrices), a block whose smallest
 // eigenvalue is not at least REDO_RATIO of the largest (this includes non-finite spectra) is queued
 // in mark_list[atomicAdd(mark_count)] for a second pass with the exact Gram matrix.
+// NT threads: D with FULL (thread t resolves lambda_{t+1}), else 64 (threads 0 .. EV_TOP - 1 resolve
+// lambda_1 .. lambda_EV_TOP, thread EV_TOP the smallest one; lam[EV_TOP .. D-2] is not written).
+template <bool FULL>
 __device__ __forceinline__ void eigvals_block(const double *__restrict__ diag, const double *__restrict__ off,
                                               double *__restrict__ lam, int blk, int *__restrict__ mark_list,
                                               int *__restrict__ mark_count) {
+    constexpr int NT = FULL ? D : 64, NWARP = NT / 32, PER = D / NT;
     __shared__ __align__(16) double2 sde[D + EV_PAD];
     __shared__ double s_e2[D];
     __shared__ double s_red[3][4];
@@ -95,33 +106,57 @@ __device__ __forceinline__ void eigvals_block(const double *__restrict__ diag, c
     __shared__ double s_pm[D];
     const int tid = threadIdx.x;
     const size_t base = static_cast<size_t>(blk) * D;
-    const double d0 = diag[base + tid];
-    const double e0 = (tid < D - 1) ? off[base + tid] : 0.0;
-    double m = fmax(fabs(d0), fabs(e0));
+    // every thread loads PER rows of the tridiagonal matrix: rows tid, tid + NT, ..
+    double dv[PER], ev[PER];
+    double m = 0.0;
+    bool nonfinite = false;
+#pragma unroll
+    for (int q = 0; q < PER; ++q) {
+        const int i = tid + NT * q;
+        dv[q] = diag[base + i];
+        ev[q] = (i < D - 1) ? off[base + i] : 0.0;
+        m = fmax(m, fmax(fabs(dv[q]), fabs(ev[q])));
+        nonfinite |= !(fabs(dv[q]) < 1e300) || !(fabs(ev[q]) < 1e300);
+    }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m = fmax(m, __shfl_xor_sync(0xffffffffu, m, o));
     if ((tid & 31) == 0) s_red[0][tid >> 5] = m;
     // a non-finite entry anywhere poisons the whole spectrum: report NaN instead of a bracket
-    const int bad = __syncthreads_or(!(fabs(d0) < 1e300) || !(fabs(e0) < 1e300));
+    const int bad = __syncthreads_or(nonfinite);
     if (bad) {
-        lam[base + tid] = nan("");
+#pragma unroll
+        for (int q = 0; q < PER; ++q) lam[base + tid + NT * q] = nan("");
         if (mark_list && tid == 0) mark_list[atomicAdd(mark_count, 1)] = blk;
         return;
     }
-    m = fmax(fmax(s_red[0][0], s_red[0][1]), fmax(s_red[0][2], s_red[0][3]));
+    m = s_red[0][0];
+#pragma unroll
+    for (int w = 1; w < NWARP; ++w) m = fmax(m, s_red[0][w]);
     if (m == 0.0) {
-        lam[base + tid] = 0.0;
+#pragma unroll
+        for (int q = 0; q < PER; ++q) lam[base + tid + NT * q] = 0.0;
         return;
     }
     const double scale = 1.0 / m;
-    const double sd = d0 * scale, se = fabs(e0 * scale);
-    s_e2[tid] = (tid < D - 1) ? fmax(se * se, EV_E2_FLOOR) : 0.0;
+#pragma unroll
+    for (int q = 0; q < PER; ++q) {
+        const int i = tid + NT * q;
+        const double se = fabs(ev[q] * scale);
+        s_e2[i] = (i < D - 1) ? fmax(se * se, EV_E2_FLOOR) : 0.0;
+    }
     __syncthreads();
-    const double se_prev = (tid > 0) ? fabs(off[base + tid - 1] * scale) : 0.0;
-    sde[tid] = make_double2(sd, (tid > 0) ? s_e2[tid - 1] : 0.0);
-    if (tid < EV_PAD) sde[D + tid] = make_double2(0.0, 0.0);
     // Gershgorin bounds of the scaled matrix
-    double glo = sd - se - se_prev, ghi = sd + se + se_prev;
+    double glo = 1e300, ghi = -1e300;
+#pragma unroll
+    for (int q = 0; q < PER; ++q) {
+        const int i = tid + NT * q;
+        const double sd = dv[q] * scale, se = fabs(ev[q] * scale);
+        const double se_prev = (i > 0) ? fabs(off[base + i - 1] * scale) : 0.0;
+        sde[i] = make_double2(sd, (i > 0) ? s_e2[i - 1] : 0.0);
+        glo = fmin(glo, sd - se - se_prev);
+        ghi = fmax(ghi, sd + se + se_prev);
+    }
+    if (tid < EV_PAD) sde[D + tid] = make_double2(0.0, 0.0);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         glo = fmin(glo, __shfl_xor_sync(0xffffffffu, glo, o));
@@ -132,8 +167,13 @@ __device__ __forceinline__ void eigvals_block(const double *__restrict__ diag, c
         s_red[2][tid >> 5] = ghi;
     }
     __syncthreads();
-    glo = fmin(fmin(s_red[1][0], s_red[1][1]), fmin(s_red[1][2], s_red[1][3]));
-    ghi = fmax(fmax(s_red[2][0], s_red[2][1]), fmax(s_red[2][2], s_red[2][3]));
+    glo = s_red[1][0];
+    ghi = s_red[2][0];
+#pragma unroll
+    for (int w = 1; w < NWARP; ++w) {
+        glo = fmin(glo, s_red[1][w]);
+        ghi = fmax(ghi, s_red[2][w]);
+    }
     glo -= 1e-10 * (fabs(glo) + 1.0);
     ghi += 1e-10 * (fabs(ghi) + 1.0);
 
@@ -144,30 +184,37 @@ __device__ __forceinline__ void eigvals_block(const double *__restrict__ diag, c
         if (geometric) return ghi * exp2(-(9.0 * 3.321928094887362 / (D - 1)) * static_cast<double>(D - 1 - t));
         return glo + (ghi - glo) * static_cast<double>(t + 1) / static_cast<double>(D);
     };
-    {
+#pragma unroll 1
+    for (int q = 0; q < PER; ++q) {
+        const int i = tid + NT * q;
         double pm;
         int pe;
-        s_cnt[tid] = sturm_eval(sde, point(tid), pm, pe);
-        s_pm[tid] = pm;
-        s_pe[tid] = pe;
+        s_cnt[i] = sturm_eval(sde, point(i), pm, pe);
+        s_pm[i] = pm;
+        s_pe[i] = pe;
     }
     __syncthreads();
-    const int target = D - 1 - tid;  // ascending index of the eigenvalue this thread brackets
+    // ascending index of the eigenvalue this thread brackets, and where it goes
+    const bool active = FULL || tid <= EV_TOP;
+    const int slot = FULL ? tid : ((tid < EV_TOP) ? tid : D - 1);   // descending position in lam
+    const int target = D - 1 - slot;
     int t = -1;                      // largest grid index with count <= target
 #pragma unroll
     for (int step = D / 2; step > 0; step >>= 1)
         if (t + step < D && s_cnt[t + step] <= target) t += step;
     double lo = point(t), hi = (t + 1 < D) ? point(t + 1) : ghi;
     if (t == D - 1) lo = hi;   // cannot happen (every eigenvalue is below the last point); keeps the bracket sane
-    // counts and p_d at both ends (ends that are not grid points carry no value)
+    // counts and p_d at both ends (ends that are not grid points carry no value).  flo / fhi steer
+    // the interpolation and may be halved (Illinois); tlo / thi stay the true values.
     int clo = (t >= 0) ? s_cnt[t] : 0, chi = (t + 1 < D) ? s_cnt[t + 1] : D;
     double flo = (t >= 0) ? s_pm[t] : 0.0, fhi = (t + 1 < D) ? s_pm[t + 1] : 0.0;
+    double tlo = flo, thi = fhi;
     int elo = (t >= 0) ? s_pe[t] : EV_PE_INVALID, ehi = (t + 1 < D) ? s_pe[t + 1] : EV_PE_INVALID;
     int replaced = 0;   // +1: the last point became hi, -1: it became lo
     int poor = 0;
     for (int it = 0; it < EV_MAX_ITER; ++it) {
         const double mid = 0.5 * (lo + hi);
-        const bool done = (hi - lo) <= fmax(2e-15, 1e-8 * fabs(mid));
+        const bool done = !active || (hi - lo) <= fmax(2e-15, 1e-8 * fabs(mid));
         if (__all_sync(0xffffffffu, done)) break;
         double x = mid;
         // p_d varies like x^d over a wide bracket, far from linear: interpolate only in a narrow one
@@ -188,6 +235,7 @@ __device__ __forceinline__ void eigvals_block(const double *__restrict__ diag, c
             hi = x;
             chi = c;
             fhi = pm;
+            thi = pm;
             ehi = pe;
             if (secant && replaced > 0) flo *= 0.5;
             replaced = 1;
@@ -195,31 +243,105 @@ __device__ __forceinline__ void eigvals_block(const double *__restrict__ diag, c
             lo = x;
             clo = c;
             flo = pm;
+            tlo = pm;
             elo = pe;
             if (secant && replaced < 0) fhi *= 0.5;
             replaced = -1;
         }
         poor = (hi - lo > 0.5 * width) ? poor + 1 : 0;   // three steps in a row that fail to halve the bracket force a bisection
     }
-    const double ev = 0.5 * (lo + hi) * m;
-    lam[base + tid] = ev;
+    // The bracket is 1e-8 wide; one more interpolation of p_d between its ends (no further
+    // evaluation) lands within the square of that of the root, which the spectral kernel's
+    // sums near a kept eigenvalue need.
+    double xr = 0.5 * (lo + hi);
+    if (chi - clo == 1 && elo > EV_PE_INVALID / 2 && ehi > EV_PE_INVALID / 2 && tlo != 0.0) {
+        const double r = scalbn(thi / tlo, max(-2000, min(2000, ehi - elo)));
+        if (r < 0.0) {
+            const double xs = lo + (hi - lo) / (1.0 - r);
+            if (xs >= lo && xs <= hi) xr = xs;
+        }
+    }
+    const double evv = xr * m;
+    if (active) lam[base + slot] = evv;
     if (mark_list) {   // uniform over the CTA
-        if (tid == 0) s_red[0][0] = ev;   // the largest eigenvalue
+        if (tid == 0) s_red[0][0] = evv;   // the largest eigenvalue
         __syncthreads();
-        if (tid == D - 1 && !(ev >= REDO_RATIO * s_red[0][0])) mark_list[atomicAdd(mark_count, 1)] = blk;
+        if (slot == D - 1 && active && !(evv >= REDO_RATIO * s_red[0][0])) mark_list[atomicAdd(mark_count, 1)] = blk;
     }
 }
 
-__global__ void __launch_bounds__(D) eigvals_kernel(const double *__restrict__ diag, const double *__restrict__ off,
-                                                    double *__restrict__ lam, const int *__restrict__ list,
-                                                    const int *__restrict__ count, int *__restrict__ mark_list,
-                                                    int *__restrict__ mark_count) {
+template <bool FULL>
+__global__ void __launch_bounds__(FULL ? D : 64) eigvals_kernel(const double *__restrict__ diag, const double *__restrict__ off,
+                                                               double *__restrict__ lam, const int *__restrict__ list,
+                                                               const int *__restrict__ count, int *__restrict__ mark_list,
+                                                               int *__restrict__ mark_count) {
     // without a list: block blockIdx.x; with one: the listed blocks, shared out over the grid
     for (int li = blockIdx.x; !list || li < *count; li += gridDim.x) {
-        eigvals_block(diag, off, lam, list ? list[li] : li, mark_list, mark_count);
+        eigvals_block<FULL>(diag, off, lam, list ? list[li] : li, mark_list, mark_count);
         if (!list) break;
         __syncthreads();   // the shared state is reused by the next listed block
     }
+}
+
+// 1 / x to about 2^-80 relative: the hardware's 20-bit estimate and two Newton steps.  Shorter than
+// the full division, which sits on the critical path of the factorisation; x is a clamped pivot,
+// far from the subnormal range the estimate flushes.
+__device__ __forceinline__ double sp_rcp(double x) {
+    double r;
+    asm("rcp.approx.ftz.f64 %0, %1;" : "=d"(r) : "d"(x));
+    double e = fma(-x, r, 1.0);
+    r = fma(r, e, r);
+    e = fma(-x, r, 1.0);
+    return fma(r, e, r);
+}
+
+// Sums over the whole spectrum from the characteristic polynomial p(x) = det(T - x I) and its first
+// two derivatives, by the three-term recurrences
+//   p_{i+1} = (d_i - x) p_i - e_{i-1}^2 p_{i-1},   p'_{i+1} = (d_i - x) p'_i - p_i - e_{i-1}^2 p'_{i-1},
+//   p''_{i+1} = (d_i - x) p''_i - 2 p'_i - e_{i-1}^2 p''_{i-1}:
+//   s1 = sum_j 1 / (lambda_j - x) = -p'/p,   s2 = sum_j 1 / (lambda_j - x)^2 = (p'/p)^2 - p''/p.
+// sde[i] = (d_i, e_{i-1}^2) as for the Sturm counts.  The six running values are brought back to
+// within range together after every group of eight rows (the ratios do not change).
+__device__ __forceinline__ void charpoly_sums(const double2 *__restrict__ sde, double x, double &s1, double &s2) {
+    double p0 = 1.0, p1 = sde[0].x - x, q0 = 0.0, q1 = -1.0, r0 = 0.0, r1 = 0.0;
+    auto row = [&](int i) {
+        const double2 de = sde[i];
+        const double t = de.x - x;
+        const double p2 = fma(t, p1, -de.y * p0);
+        const double q2 = fma(t, q1, fma(-de.y, q0, -p1));
+        const double r2 = fma(t, r1, fma(-de.y, r0, -2.0 * q1));
+        p0 = p1;
+        p1 = p2;
+        q0 = q1;
+        q1 = q2;
+        r0 = r1;
+        r1 = r2;
+    };
+    auto rescale = [&]() {
+        const int e0 = (__double2hiint(p0) >> 20) & 0x7ff, e1 = (__double2hiint(p1) >> 20) & 0x7ff;
+        const int em = max(e0, e1);
+        if (em > 0 && em < 2047) {
+            const double sc = __hiloint2double((2046 - em) << 20, 0);   // 2^(1023 - em)
+            p0 *= sc;
+            p1 *= sc;
+            q0 *= sc;
+            q1 *= sc;
+            r0 *= sc;
+            r1 *= sc;
+        }
+    };
+    constexpr int NG = (D - 1) / 8;
+#pragma unroll 1
+    for (int g = 0; g < NG; ++g) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) row(1 + 8 * g + i);
+        rescale();
+    }
+#pragma unroll
+    for (int i = 1 + 8 * NG; i < D; ++i) row(i);
+    const double ip = sp_rcp(p1);
+    s1 = -q1 * ip;
+    s2 = fma(s1, s1, -r1 * ip);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -236,98 +358,136 @@ constexpr int LU_LANES = 12;
 static_assert(KPILOT < LU_LANES && KPILOT <= 3 * SP_WARPS, "one LU column and one warp slot per kept vector");
 constexpr size_t SPECTRAL_DYN_SMEM = sizeof(double) * 4 * D * LU_LANES;
 
-// 1 / x to about 2^-80 relative: the hardware's 20-bit estimate and two Newton steps.  Shorter than
-// the full division, which sits on the critical path of the factorisation; x is a clamped pivot,
-// far from the subnormal range the estimate flushes.
-__device__ __forceinline__ double sp_rcp(double x) {
-    double r;
-    asm("rcp.approx.ftz.f64 %0, %1;" : "=d"(r) : "d"(x));
-    double e = fma(-x, r, 1.0);
-    r = fma(r, e, r);
-    e = fma(-x, r, 1.0);
-    return fma(r, e, r);
+// Back-transformation x = H_0 H_1 ... H_{D-3} y of the kept vectors, normalisation, and the stores of
+// the right singular vectors.  The reflectors (rows of R, 1 KB each) are staged through shared memory
+// by the CTA's last warp, sixteen rows per stage and two stages, handed over with named barriers.
+// The other three warps apply them: a group of eight lanes owns one vector (sixteen entries per
+// lane: rows 16 m + 2 sub, + 1), so a dot product needs three shuffle stages and four vectors share
+// every instruction.  Reflector k is zero up to index k, and whole 16-row chunks of zeros are skipped.
+constexpr int BT_ROWS = 16;                 // reflector rows per stage
+constexpr int BT_BAR_FULL = 2, BT_BAR_EMPTY = 4;   // named barriers: + stage
+static_assert(2 * BT_ROWS * D <= 3 * D * LU_LANES, "the ring reuses the storage of the factorisations");
+
+// (barrier numbers are spelled out: a number in a register makes the compiler reserve all sixteen)
+__device__ __forceinline__ void bt_bar_sync(int id) {
+    if (id == 2) asm volatile("bar.sync 2, 128;" ::: "memory");
+    else if (id == 3) asm volatile("bar.sync 3, 128;" ::: "memory");
+    else if (id == 4) asm volatile("bar.sync 4, 128;" ::: "memory");
+    else asm volatile("bar.sync 5, 128;" ::: "memory");
+}
+__device__ __forceinline__ void bt_bar_arrive(int id) {
+    if (id == 2) asm volatile("bar.arrive 2, 128;" ::: "memory");
+    else if (id == 3) asm volatile("bar.arrive 3, 128;" ::: "memory");
+    else if (id == 4) asm volatile("bar.arrive 4, 128;" ::: "memory");
+    else asm volatile("bar.arrive 5, 128;" ::: "memory");
 }
 
-// Back-transformation of the NV vectors warp, warp + 4, .. of `yv` through the reflectors stored in
-// the rows of R, normalisation, and the stores of the kept right singular vectors.
-// Reflectors are applied two at a time, H_{k-1} H_k y = y - g_k u_k - g_{k-1} u_{k-1} with
-//   g_k = t_k (u_k . y),   g_{k-1} = t_{k-1} ((u_{k-1} . y) - g_k (u_{k-1} . u_k)),
-// so that one round of warp reductions serves two steps, and their rows are fetched from global
-// memory two pairs ahead of use.
-template <int NV>
 __device__ __forceinline__ void sp_back_transform(const double *__restrict__ R, const double *__restrict__ tt,
-                                                  const double *__restrict__ yv, int warp, int lane, float *__restrict__ vr,
-                                                  const eosq_cache_t &out, long long gb) {
-    double y[NV][4];
-#pragma unroll
-    for (int v = 0; v < NV; ++v)
-#pragma unroll
-        for (int m = 0; m < 4; ++m) y[v][m] = yv[(lane + 32 * m) * LU_LANES + warp + SP_WARPS * v];
-    double ring[2][2][4];
-    auto load_pair = [&](int k, double (&dst)[2][4]) {
-#pragma unroll
-        for (int m = 0; m < 4; ++m) {
-            dst[0][m] = __ldg(R + static_cast<size_t>(k) * D + lane + 32 * m);
-            dst[1][m] = __ldg(R + static_cast<size_t>(k - 1) * D + lane + 32 * m);
-        }
-    };
-    load_pair(D - 3, ring[0]);
-    load_pair(D - 5, ring[1]);
+                                                  const double *__restrict__ yv, double *__restrict__ ring, int rank, int warp,
+                                                  int lane, float *__restrict__ vr, const eosq_cache_t &out, long long gb) {
+    constexpr int NSTAGE = (D - 2 + BT_ROWS - 1) / BT_ROWS;
+    double2 *ring2 = reinterpret_cast<double2 *>(ring);
+    if (warp == SP_WARPS - 1) {
+        // producer: rows klo .. khi of R are contiguous in global memory
+        const double2 *R2 = reinterpret_cast<const double2 *>(R);
 #pragma unroll 1
-    for (int k0 = D - 3; k0 >= 1; k0 -= 4) {
+        for (int j = 0; j < NSTAGE; ++j) {
+            const int st = j & 1;
+            const int khi = D - 3 - BT_ROWS * j, klo = max(khi - (BT_ROWS - 1), 0);
+            const int cnt2 = (khi - klo + 1) * (D / 2);
+            if (j >= 2) bt_bar_sync(BT_BAR_EMPTY + st);
+            const double2 *src = R2 + static_cast<size_t>(klo) * (D / 2);
+            double2 *dst = ring2 + st * (BT_ROWS * D / 2);
+#pragma unroll 1
+            for (int e0 = 0; e0 < cnt2; e0 += 32 * 8) {
+                double2 v[8];
 #pragma unroll
-        for (int s2 = 0; s2 < 2; ++s2) {
-            const int k = k0 - 2 * s2;
-            if (k >= 1) {
-                double ua[4], ub[4];
-#pragma unroll
-                for (int m = 0; m < 4; ++m) {
-                    ua[m] = ring[s2][0][m];
-                    ub[m] = ring[s2][1][m];
+                for (int q = 0; q < 8; ++q) {
+                    const int e = e0 + 32 * q + lane;
+                    v[q] = (e < cnt2) ? __ldg(src + e) : make_double2(0.0, 0.0);
                 }
-                if (k - 4 >= 1) load_pair(k - 4, ring[s2]);
-                const double ta = tt[k], tb = tt[k - 1];
-                double dots[2 * NV + 1];
 #pragma unroll
-                for (int v = 0; v < NV; ++v) {
-                    dots[2 * v] = fma(ua[0], y[v][0], ua[1] * y[v][1]) + fma(ua[2], y[v][2], ua[3] * y[v][3]);
-                    dots[2 * v + 1] = fma(ub[0], y[v][0], ub[1] * y[v][1]) + fma(ub[2], y[v][2], ub[3] * y[v][3]);
+                for (int q = 0; q < 8; ++q) {
+                    const int e = e0 + 32 * q + lane;
+                    if (e < cnt2) dst[e] = v[q];
                 }
-                dots[2 * NV] = fma(ua[0], ub[0], ua[1] * ub[1]) + fma(ua[2], ub[2], ua[3] * ub[3]);
+            }
+            bt_bar_arrive(BT_BAR_FULL + st);
+        }
+        return;
+    }
+    const int grp = lane >> 3, sub = lane & 7;
+    const int vi = 4 * warp + grp;
+    const bool live = vi < rank;
+    double y[16];
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1)
+    for (int m = 0; m < 8; ++m) {
+        y[2 * m] = live ? yv[(16 * m + 2 * sub) * LU_LANES + vi] : 0.0;
+        y[2 * m + 1] = live ? yv[(16 * m + 2 * sub + 1) * LU_LANES + vi] : 0.0;
+    }
+#pragma unroll 1
+    for (int j = 0; j < NSTAGE; ++j) {
+        const int st = j & 1;
+        const int khi = D - 3 - BT_ROWS * j, klo = max(khi - (BT_ROWS - 1), 0);
+        bt_bar_sync(BT_BAR_FULL + st);
+        if (4 * warp < rank) {   // a warp without vectors only keeps the barriers going
+            const double2 *stage = ring2 + st * (BT_ROWS * D / 2);
+#pragma unroll 1
+            for (int k = khi; k >= klo; --k) {
+                const double2 *urow = stage + (k - klo) * (D / 2) + sub;
+                const int m0 = (k + 1) >> 4;   // chunks below it hold only zeros of the reflector
+                double2 u[8];
+                double d0 = 0.0, d1 = 0.0;
 #pragma unroll
-                    for (int q = 0; q < 2 * NV + 1; ++q) dots[q] += __shfl_xor_sync(0xffffffffu, dots[q], o);
+                for (int m = 0; m < 8; ++m) {
+                    if (m >= m0) {
+                        u[m] = urow[8 * m];
+                        d0 = fma(u[m].x, y[2 * m], d0);
+                        d1 = fma(u[m].y, y[2 * m + 1], d1);
+                    }
+                }
+                double dot = d0 + d1;
+                dot += __shfl_xor_sync(0xffffffffu, dot, 1);
+                dot += __shfl_xor_sync(0xffffffffu, dot, 2);
+                dot += __shfl_xor_sync(0xffffffffu, dot, 4);
+                const double g = tt[k] * dot;
 #pragma unroll
-                for (int v = 0; v < NV; ++v) {
-                    const double ga = ta * dots[2 * v];
-                    const double gbb = tb * fma(-ga, dots[2 * NV], dots[2 * v + 1]);
-#pragma unroll
-                    for (int m = 0; m < 4; ++m) y[v][m] = fma(-gbb, ub[m], fma(-ga, ua[m], y[v][m]));
+                for (int m = 0; m < 8; ++m) {
+                    if (m >= m0) {
+                        y[2 * m] = fma(-g, u[m].x, y[2 * m]);
+                        y[2 * m + 1] = fma(-g, u[m].y, y[2 * m + 1]);
+                    }
                 }
             }
         }
+        if (j + 2 < NSTAGE) bt_bar_arrive(BT_BAR_EMPTY + st);
     }
+    double nn = 0.0;
 #pragma unroll
-    for (int v = 0; v < NV; ++v) {
-        const int vi = warp + SP_WARPS * v;
-        double nn = fma(y[v][0], y[v][0], y[v][1] * y[v][1]) + fma(y[v][2], y[v][2], y[v][3] * y[v][3]);
-        nn = warp_sum(nn);
-        const double rn = (nn > 0.0) ? rsqrt(nn) : 0.0;
+    for (int e = 0; e < 16; ++e) nn = fma(y[e], y[e], nn);
+    nn += __shfl_xor_sync(0xffffffffu, nn, 1);
+    nn += __shfl_xor_sync(0xffffffffu, nn, 2);
+    nn += __shfl_xor_sync(0xffffffffu, nn, 4);
+    const double rn = (nn > 0.0) ? rsqrt(nn) : 0.0;
+    if (live) {
 #pragma unroll
-        for (int m = 0; m < 4; ++m) {
-            const int j = lane + 32 * m;
-            const float f = static_cast<float>(y[v][m] * rn);
-            vr[vi * D + j] = f;
-            out.V[(gb * RMAX + vi) * D + j] = __half_as_ushort(__float2half_rn(f));
-            if (out.vr32) out.vr32[(gb * RMAX + vi) * D + j] = f;
+        for (int m = 0; m < 8; ++m) {
+            const int jrow = 16 * m + 2 * sub;
+            const float f0 = static_cast<float>(y[2 * m] * rn), f1 = static_cast<float>(y[2 * m + 1] * rn);
+            *reinterpret_cast<float2 *>(vr + vi * D + jrow) = make_float2(f0, f1);
+            *reinterpret_cast<uint32_t *>(out.V + (gb * RMAX + vi) * D + jrow) =
+                static_cast<uint32_t>(__half_as_ushort(__float2half_rn(f0))) | (static_cast<uint32_t>(__half_as_ushort(__float2half_rn(f1))) << 16);
+            if (out.vr32) *reinterpret_cast<float2 *>(out.vr32 + (gb * RMAX + vi) * D + jrow) = make_float2(f0, f1);
         }
     }
 }
 
-__global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspace ws, eosq_cache_t out, long long block0) {
+__global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspace ws, eosq_cache_t out, long long block0, bool full) {
     __shared__ double lam[D], dd[D], ee[D], tt[D], atoms[D];
     __shared__ double inv_e[D];              // reciprocals of the (clamped) subdiagonal entries
+    __shared__ __align__(16) double2 sde[D];  // (d_i, e_{i-1}^2) of the scaled matrix, for the characteristic polynomial
+    __shared__ double st1[6 * KPILOT], st2[6 * KPILOT];   // weighted samples of the tail sums around each kept eigenvalue
+    __shared__ double s_max[SP_WARPS];
     __shared__ double s_phi[RMAX], s_sig[RMAX];
     __shared__ unsigned s_flags;
     extern __shared__ double dyn[];
@@ -340,11 +500,16 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
     const int b = blockIdx.x;
     const long long gb = block0 + b;
     const size_t base = static_cast<size_t>(b) * D;
-    if (tid < D) {
-        lam[tid] = ws.lam[base + tid];
+    {
+        // lam[EV_TOP .. D-2] holds eigenvalues only when the full spectrum was asked for
+        lam[tid] = (full || tid < EV_TOP || tid == D - 1) ? ws.lam[base + tid] : 0.0;
         dd[tid] = ws.diag[base + tid];
         ee[tid] = ws.off[base + tid];
         tt[tid] = ws.tau[base + tid];
+        double mx = fmax(fabs(dd[tid]), fabs(ee[tid]));
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mx = fmax(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        if (lane == 0) s_max[warp] = mx;
     }
     if (tid < RMAX) {
         s_phi[tid] = 0.0;
@@ -352,12 +517,13 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
     }
     if (tid == 0) s_flags = 0u;
     __syncthreads();
+    const double mscale = fmax(fmax(s_max[0], s_max[1]), fmax(s_max[2], s_max[3]));
 
     // Step 1: bulk edge from lambda_{k+1}, lambda_{2k+1} (1-based) and the rank test.
     const double edge_c = 1.0 / (cbrt(4.0) - 1.0);
     const double cut = 1.0 / cbrt(static_cast<double>(D));
     const double lam_plus = lam[KPILOT] + edge_c * (lam[KPILOT] - lam[2 * KPILOT]);
-    const bool pass = (tid < D) && (lam[tid] / lam_plus - 1.0 > cut);
+    const bool pass = (tid < EV_TOP) && (lam[tid] / lam_plus - 1.0 > cut);
     int rank = __syncthreads_count(pass);
     if (tid == 0) {
         unsigned f = 0u;
@@ -368,11 +534,12 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
     if (rank > KPILOT) rank = KPILOT;
 
     if (rank > 0) {
-        // Step 2: k imputed atoms behind the outliers, observed eigenvalues after them.
-        if (tid < D) {
+        // Step 2: k imputed atoms behind the outliers; the observed eigenvalues after them are known
+        // one by one up to lambda_EV_TOP, the rest (the tail) only through sums.
+        {
             double a = 0.0;
-            if (tid >= rank + KPILOT) a = lam[tid];
-            else if (tid >= rank) {
+            if (tid >= rank + KPILOT && tid < EV_TOP) a = lam[tid];
+            else if (tid >= rank && tid < rank + KPILOT) {
                 const int jj = tid - rank + 1;
                 const double bs = lam[KPILOT + rank];
                 const double gap = bs - lam[2 * KPILOT + rank];
@@ -381,47 +548,89 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
             atoms[tid] = a;
         }
         const double floor_piv = 1.2e-16 * fmax(fabs(lam[0]), 1e-300);
-        if (tid < D) {   // pivots taken from the subdiagonal do not depend on the vector: their reciprocals are shared
+        {   // pivots taken from the subdiagonal do not depend on the vector: their reciprocals are shared
             double l = ee[tid];
             if (!(fabs(l) >= floor_piv)) l = (l < 0.0) ? -floor_piv : floor_piv;
             inv_e[tid] = sp_rcp(l);
+            const double is = (mscale > 0.0) ? 1.0 / mscale : 0.0;
+            const double se = (tid > 0) ? fabs(ee[tid - 1] * is) : 0.0;
+            sde[tid] = make_double2(dd[tid] * is, (tid > 0) ? fmax(se * se, EV_E2_FLOOR) : 0.0);
         }
         __syncthreads();
-        // Step 3: Stieltjes transforms of F_e at z = lambda_i, D-transform, Eq. 9, Eq. 6.
-        for (int i = warp; i < rank; i += SP_WARPS) {
-            const double z = lam[i];
-            double ms = 0.0, msp = 0.0;
-            for (int j = rank + lane; j < D; j += 32) {
-                const double inv = 1.0 / (atoms[j] - z);
-                ms += inv;
-                msp += inv * inv;
-            }
-            ms = warp_sum(ms);
-            msp = warp_sum(msp);
-            if (lane == 0) {
-                const double nn = static_cast<double>(D - rank);
-                ms /= nn;
-                msp /= nn;
-                const double ratio = static_cast<double>(D) / static_cast<double>(n);
-                const double m1 = ratio * ms - (1.0 - ratio) / z;  // n x n side: n - d extra zeros
-                const double m1p = ratio * msp + (1.0 - ratio) / (z * z);
-                const double m2 = ms, m2p = msp;                   // d x d side
-                const double T = z * m1 * m2;
-                const double Tp = m1 * m2 + z * (m1p * m2 + m1 * m2p);
-                const double dh = 1.0 / sqrt(T);
-                const double a1 = m1 / (dh * dh * Tp), a2 = m2 / (dh * dh * Tp);
-                double ph = dh * sqrt(a1 * a2);
-                const double sg = sqrt(z);
-                if (!(ph >= 0.0) || !(ph < 1e300)) {
-                    ph = 0.0;
-                    atomicOr(&s_flags, EOSQ_BLOCK_CLAMPED);
-                } else if (ph > sg) {
-                    ph = sg;
-                    atomicOr(&s_flags, EOSQ_BLOCK_CLAMPED);
+        // Tail sums  sum_{j > EV_TOP} 1 / (lambda_j - z)  and  sum 1 / (lambda_j - z)^2  at z = lambda_i:
+        // the sums over the whole spectrum have a pole at z, so they are taken at six points
+        // z + m h, m = -3 .. 3 without 0, the known eigenvalues are subtracted there, and what is left
+        // (smooth: the tail lies well below z) is interpolated to z, exact for polynomials of degree 5.
+        // h = z / 64, or less when a neighbouring known eigenvalue is closer than 3.5 h.
+        // Warps 1 .. 3 take these sums and Step 3 while warp 0 factorises for the eigenvectors below.
+        if (warp > 0) {
+            const int e = tid - 32;
+            if (e < 6 * rank) {
+                const int i = e / 6, m6 = e % 6;
+                const int mm = (m6 < 3) ? m6 - 3 : m6 - 2;   // -3, -2, -1, 1, 2, 3
+                const double z = lam[i];
+                double gnn = z - lam[i + 1];
+                if (i > 0) gnn = fmin(gnn, lam[i - 1] - z);
+                const double h = fmin(z * (1.0 / 64.0), gnn * (1.0 / 3.5));
+                const double x = fma(static_cast<double>(mm), h, z);
+                const double is = sp_rcp(mscale);
+                double f1, f2;
+                charpoly_sums(sde, x * is, f1, f2);
+                f1 *= is;
+                f2 *= is * is;
+#pragma unroll 2
+                for (int j = 0; j < EV_TOP; ++j) {
+                    const double inv = sp_rcp(lam[j] - x);
+                    f1 -= inv;
+                    f2 = fma(-inv, inv, f2);
                 }
-                s_phi[i] = ph;
-                s_sig[i] = sg;
-                if (i > 0 && (lam[i - 1] - z) < 1e-9 * lam[i - 1]) atomicOr(&s_flags, EOSQ_BLOCK_CLUSTERED);
+                const int am = (mm < 0) ? -mm : mm;
+                const double w = (am == 1) ? 15.0 / 20.0 : ((am == 2) ? -6.0 / 20.0 : 1.0 / 20.0);
+                st1[e] = w * f1;
+                st2[e] = w * f2;
+                if (!(h > z * (1.0 / 16384.0))) atomicOr(&s_flags, EOSQ_BLOCK_CLUSTERED);
+            }
+            asm volatile("bar.sync 1, 96;" ::: "memory");
+            // Step 3: Stieltjes transforms of F_e at z = lambda_i, D-transform, Eq. 9, Eq. 6.
+            for (int i = warp - 1; i < rank; i += SP_WARPS - 1) {
+                const double z = lam[i];
+                double ms = 0.0, msp = 0.0;
+                for (int j = rank + lane; j < EV_TOP; j += 32) {
+                    const double inv = sp_rcp(atoms[j] - z);
+                    ms += inv;
+                    msp = fma(inv, inv, msp);
+                }
+                if (lane < 6) {
+                    ms += st1[6 * i + lane];
+                    msp += st2[6 * i + lane];
+                }
+                ms = warp_sum(ms);
+                msp = warp_sum(msp);
+                if (lane == 0) {
+                    const double nn = static_cast<double>(D - rank);
+                    ms /= nn;
+                    msp /= nn;
+                    const double ratio = static_cast<double>(D) / static_cast<double>(n);
+                    const double m1 = ratio * ms - (1.0 - ratio) / z;  // n x n side: n - d extra zeros
+                    const double m1p = ratio * msp + (1.0 - ratio) / (z * z);
+                    const double m2 = ms, m2p = msp;                   // d x d side
+                    const double T = z * m1 * m2;
+                    const double Tp = m1 * m2 + z * (m1p * m2 + m1 * m2p);
+                    const double dh = 1.0 / sqrt(T);
+                    const double a1 = m1 / (dh * dh * Tp), a2 = m2 / (dh * dh * Tp);
+                    double ph = dh * sqrt(a1 * a2);
+                    const double sg = sqrt(z);
+                    if (!(ph >= 0.0) || !(ph < 1e300)) {
+                        ph = 0.0;
+                        atomicOr(&s_flags, EOSQ_BLOCK_CLAMPED);
+                    } else if (ph > sg) {
+                        ph = sg;
+                        atomicOr(&s_flags, EOSQ_BLOCK_CLAMPED);
+                    }
+                    s_phi[i] = ph;
+                    s_sig[i] = sg;
+                    if (i > 0 && (lam[i - 1] - z) < 1e-9 * lam[i - 1]) atomicOr(&s_flags, EOSQ_BLOCK_CLUSTERED);
+                }
             }
         }
 
@@ -590,16 +799,11 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
     }
     __syncthreads();
 
-    // Back-transformation x = H_0 H_1 ... H_{D-3} y; warp w takes those of the vectors w, w + 4, w + 8
-    // that exist (the instruction count follows the number of vectors, so it is a template argument).
+    // Back-transformation of the kept vectors (the ring takes the place of the factorisations, which
+    // are no longer needed after the barrier above).
     const double *R = ws.gram + static_cast<size_t>(b) * D * D;
     float *vr = ws.vr + static_cast<size_t>(b) * RMAX * D;
-    if (warp < rank) {
-        const int nv = (rank - warp + SP_WARPS - 1) / SP_WARPS;
-        if (nv == 1) sp_back_transform<1>(R, tt, yv, warp, lane, vr, out, gb);
-        else if (nv == 2) sp_back_transform<2>(R, tt, yv, warp, lane, vr, out, gb);
-        else sp_back_transform<3>(R, tt, yv, warp, lane, vr, out, gb);
-    }
+    if (rank > 0) sp_back_transform(R, tt, yv, dyn, rank, warp, lane, vr, out, gb);
     // rows >= rank of V are zero; scalars
     for (int e = tid; e < RMAX * D; e += SP_THREADS) {
         if (e / D >= rank) {
@@ -617,7 +821,7 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
         ws.coef[static_cast<size_t>(b) * RMAX + tid] = cf;
         if (out.coef) out.coef[gb * RMAX + tid] = cf;
     }
-    if (tid < D && out.eig) out.eig[gb * D + tid] = static_cast<float>(lam[tid]);
+    if (full && out.eig) out.eig[gb * D + tid] = static_cast<float>(lam[tid]);
     if (tid == 0) {
         if (b == 0) *ws.redo_count = 0;   // the second pass of this chunk is over: empty its queue for the next chunk
         out.rank[gb] = rank;
@@ -627,11 +831,12 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
     }
 }
 
-void launch_eigvals(int64_t nb, const Workspace &ws, const int *list, const int *count, int *mark_list, cudaStream_t s) {
-    eigvals_kernel<<<list_grid(nb, list), D, 0, s>>>(ws.diag, ws.off, ws.lam, list, count, mark_list, ws.redo_count);
+void launch_eigvals(int64_t nb, const Workspace &ws, const int *list, const int *count, int *mark_list, bool full, cudaStream_t s) {
+    if (full) eigvals_kernel<true><<<list_grid(nb, list), D, 0, s>>>(ws.diag, ws.off, ws.lam, list, count, mark_list, ws.redo_count);
+    else eigvals_kernel<false><<<list_grid(nb, list), 64, 0, s>>>(ws.diag, ws.off, ws.lam, list, count, mark_list, ws.redo_count);
 }
 
-void launch_spectral(int64_t nb, int n, const Workspace &ws, const eosq_cache_t &out, int64_t block0,
+void launch_spectral(int64_t nb, int n, const Workspace &ws, const eosq_cache_t &out, int64_t block0, bool full,
                      cudaStream_t s) {
     static bool configured = false;
     if (!configured) {
@@ -639,7 +844,7 @@ void launch_spectral(int64_t nb, int n, const Workspace &ws, const eosq_cache_t 
                              static_cast<int>(SPECTRAL_DYN_SMEM));
         configured = true;
     }
-    spectral_kernel<<<static_cast<unsigned>(nb), SP_THREADS, SPECTRAL_DYN_SMEM, s>>>(n, ws, out, static_cast<long long>(block0));
+    spectral_kernel<<<static_cast<unsigned>(nb), SP_THREADS, SPECTRAL_DYN_SMEM, s>>>(n, ws, out, static_cast<long long>(block0), full);
 }
 
 }  // namespace eosq
