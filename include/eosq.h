@@ -106,7 +106,8 @@ size_t eosq_workspace_bytes(int64_t num_blocks, int n, int d);
 
 /* Create / destroy a context on the current device.  The context lazily builds and caches, per
  * (d, seed) and (d, bits), the device copies of Pi and of the codebook; building one performs a
- * synchronous host-to-device copy on first use.  Not thread safe. */
+ * synchronous host-to-device copy on first use.  Not thread safe.  Every device entry point below
+ * returns EOSQ_ERR_INVALID_ARG when the current CUDA device is not the context's. */
 int eosq_create(eosq_ctx **out);
 int eosq_destroy(eosq_ctx *ctx);
 
@@ -147,8 +148,11 @@ int eosq_encode(eosq_ctx *ctx, const void *blocks, int in_dtype, int64_t num_blo
  *   - num_blocks <= EOSQ_STATIC_MAX_BLOCKS; a larger count is rejected with
  *     EOSQ_ERR_BUFFER_TOO_SMALL (text in eosq_last_cuda_error) and nothing is enqueued.
  *   - The first call on a device looks up the array's device address (that device must be
- *     current, as for every call), and the first call with a new seed uploads that seed's
- *     rotation from host memory on the given stream.  Make those calls before any stream capture.
+ *     current and must be the context's device, as for every call), the first call with a new seed
+ *     uploads that seed's rotation from host memory on the given stream, and the first call with a
+ *     new (in_dtype, bits) pair on a device loads those kernels and sets their shared-memory
+ *     limits.  Make those calls before any stream capture, and keep per-stage profiling off
+ *     (eosq_profile_enable creates events on first use).
  *   - All calls on a device share the one array, and it keeps whatever the last call left.  The
  *     kernels write every scratch value before reading it, so nothing needs clearing, but two
  *     calls that overlap on the GPU (different streams, no ordering between them) race; order
@@ -163,10 +167,10 @@ int eosq_encode_static(eosq_ctx *ctx, const void *blocks, int in_dtype, int64_t 
  * Reconstruct blocks from a compressed cache (Algorithm 1 last TQ_MSE line, Algorithm 2 Return):
  *   x_hat[t] = sum_{i<r} P[i][t] V[i][:] + norms[t] * Pi^T centroids[codes[t]].
  *   out_blocks dev [num_blocks][n][d] of out_dtype (EOSQ_F16 or EOSQ_F32).
- * With codes, norms, P and out_blocks 16-byte aligned the tensor-core kernel runs; it (and the score
- * kernel) reads at most 12 factor rows per block (eosq_encode stores at most the pilot k = 11), so a
- * cache written elsewhere with a larger rank word is truncated to 12.  Other layouts take a slower
- * CUDA-core kernel.
+ * codes, norms, P and out_blocks must be 16-byte aligned (EOSQ_ERR_INVALID_ARG otherwise: the
+ * kernel moves them with bulk copies and tensor stores).  It (and the score kernel) reads at most
+ * 12 factor rows per block (eosq_encode stores at most the pilot k = 11), so a cache written
+ * elsewhere with a larger rank word is truncated to 12.
  */
 int eosq_decode(eosq_ctx *ctx, const eosq_cache_t *cache, int64_t num_blocks, int n, int d, int bits,
                 uint64_t seed, void *out_blocks, int out_dtype, void *cuda_stream);
@@ -180,6 +184,7 @@ int eosq_decode(eosq_ctx *ctx, const eosq_cache_t *cache, int64_t num_blocks, in
  * out [head][K|V][block]).
  *   q       dev [num_kv_heads][G][d] fp16
  *   scores  dev [num_kv_heads][G][blocks_per_head*n] fp32
+ * codes, norms, P and V of `kcache` must be 16-byte aligned (EOSQ_ERR_INVALID_ARG otherwise).
  * The tensor-core path keeps the rotated queries in a device buffer of 4 KB per KV head that the
  * context owns: the first call (and a later call with more heads) allocates it, which synchronises
  * the device; calls on one context must not overlap in time.
@@ -215,11 +220,11 @@ int64_t eosq_launch_count(const eosq_ctx *ctx);
  * CUDA events on the launching stream.  eosq_profile_read synchronises those events, adds their
  * elapsed milliseconds into ms[EOSQ_NUM_STAGES] and their launch counts into
  * launches[EOSQ_NUM_STAGES] (host arrays, overwritten), and clears the record.
- * Stage order: Gram, tridiagonalisation steps 0-31, 32-63 and 64-125 (three kernels), eigenvalues,
+ * Stage order: Gram, tridiagonalisation steps 0-63 and 64-125 (two kernels), eigenvalues,
  * spectrum + shrinkage + eigenvectors, residual/rotate/quantise/pack, decode, scores, the second
  * pass over blocks whose tensor-core Gram matrix was not accurate enough (all its kernels), other.
  */
-#define EOSQ_NUM_STAGES 11
+#define EOSQ_NUM_STAGES 10
 int eosq_profile_enable(eosq_ctx *ctx, int on);
 /* Times only the stages whose bit (1 << stage index, in the order above) is set in stage_mask; the
  * two events per launch cost about 2 us of device time each, which adds up over the several hundred

@@ -3,12 +3,38 @@
 #include <algorithm>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
+#include <utility>
 
 #include "eosq_common.cuh"
 
 using namespace eosq;
 
+bool eosq::ensure_dynamic_smem(const void *kernel, size_t bytes) {
+    static std::mutex mu;
+    static std::vector<std::pair<const void *, int>> done;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    std::lock_guard<std::mutex> lock(mu);
+    for (const auto &e : done)
+        if (e.first == kernel && e.second == dev) return true;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes)) != cudaSuccess) return false;
+    done.emplace_back(kernel, dev);
+    return true;
+}
+
 namespace {
+
+// The context's buffers, constants and error word live on the device it was created on: every
+// device entry point refuses to run with another device current.
+bool on_ctx_device(eosq_ctx *ctx) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev != ctx->device) {
+        ctx->last_error = "the current CUDA device is not the one this context was created on";
+        return false;
+    }
+    return true;
+}
 
 bool record_cuda(eosq_ctx *ctx, cudaError_t err, const char *what) {
     if (err == cudaSuccess) return false;
@@ -255,7 +281,7 @@ extern "C" int eosq_encode(eosq_ctx *ctx, const void *blocks, int in_dtype, int6
     int rc = check_shape(n, d, bits);
     if (rc != EOSQ_OK) return rc;
     if (num_blocks == 0) return EOSQ_OK;
-    if (!blocks || !cache_required_ok(out) || !workspace) return EOSQ_ERR_INVALID_ARG;
+    if (!blocks || !cache_required_ok(out) || !workspace || !on_ctx_device(ctx)) return EOSQ_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(blocks) & 15u) || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
         (reinterpret_cast<uintptr_t>(out->codes) & 15u))
         return EOSQ_ERR_INVALID_ARG;
@@ -283,22 +309,21 @@ extern "C" int eosq_decode(eosq_ctx *ctx, const eosq_cache_t *cache, int64_t num
     int rc = check_shape(n, d, bits);
     if (rc != EOSQ_OK) return rc;
     if (num_blocks == 0) return EOSQ_OK;
-    if (!cache || !cache->codes || !cache->norms || !cache->rank || !cache->P || !cache->V || !out_blocks)
+    if (!cache || !cache->codes || !cache->norms || !cache->rank || !cache->P || !cache->V || !out_blocks || !on_ctx_device(ctx))
         return EOSQ_ERR_INVALID_ARG;
     Rotation rot;
     Codebook cb;
     if ((rc = get_rotation(ctx, d, seed, &rot)) != EOSQ_OK) return rc;
     if ((rc = get_codebook(d, bits, &cb)) != EOSQ_OK) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    if (decode_tc_supported(*cache, bits, out_blocks)) {
+    if (!decode_tc_supported(*cache, bits, out_blocks)) return EOSQ_ERR_INVALID_ARG;   // 16-byte alignment of codes, norms, P, out_blocks
+    {
         bool setup_ok = true;
         run_stage(ctx, ST_DECODE, s, [&] { setup_ok = launch_decode_tc(*cache, num_blocks, n, rot, cb, out_blocks, out_dtype, ctx->dev_err, ctx->sm_count, s); });
         if (!setup_ok) {
             ctx->last_error = "tensor-core decode kernel: launch set-up failed";
             return EOSQ_ERR_CUDA;
         }
-    } else {
-        run_stage(ctx, ST_DECODE, s, [&] { launch_decode_plain(*cache, num_blocks, n, rot, cb, out_blocks, out_dtype, s); });
     }
     if (record_cuda(ctx, cudaGetLastError(), "eosq_decode launch")) return EOSQ_ERR_CUDA;
     return EOSQ_OK;
@@ -312,15 +337,15 @@ extern "C" int eosq_scores(eosq_ctx *ctx, const eosq_cache_t *kcache, int64_t nu
     int rc = check_shape(n, d, bits);
     if (rc != EOSQ_OK) return rc;
     if (num_kv_heads == 0 || blocks_per_head == 0) return EOSQ_OK;
-    if (!kcache || !kcache->codes || !kcache->norms || !kcache->rank || !kcache->P || !kcache->V || !q || !scores)
+    if (!kcache || !kcache->codes || !kcache->norms || !kcache->rank || !kcache->P || !kcache->V || !q || !scores || !on_ctx_device(ctx))
         return EOSQ_ERR_INVALID_ARG;
-    if (reinterpret_cast<uintptr_t>(kcache->codes) & 3u) return EOSQ_ERR_INVALID_ARG;
+    if (!scores_tc_supported(*kcache, bits, n)) return EOSQ_ERR_INVALID_ARG;   // 16-byte alignment of codes, norms, P, V
     Rotation rot;
     Codebook cb;
     if ((rc = get_rotation(ctx, d, seed, &rot)) != EOSQ_OK) return rc;
     if ((rc = get_codebook(d, bits, &cb)) != EOSQ_OK) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    if (scores_tc_supported(*kcache, bits, n) && (reinterpret_cast<uintptr_t>(kcache->codes) & 15u) == 0) {
+    {
         bool setup_ok = true;
         int64_t kernels = 0;
         run_stage(ctx, ST_SCORES, s, [&] {
@@ -333,11 +358,6 @@ extern "C" int eosq_scores(eosq_ctx *ctx, const eosq_cache_t *kcache, int64_t nu
             ctx->last_error = "tensor-core score kernel: launch set-up failed";
             return EOSQ_ERR_CUDA;
         }
-    } else {
-        run_stage(ctx, ST_SCORES, s, [&] {
-            launch_scores_plain(*kcache, num_kv_heads, blocks_per_head, head_stride_blocks, n, rot, cb,
-                                static_cast<const __half *>(q), G, scale, scores, s);
-        });
     }
     if (record_cuda(ctx, cudaGetLastError(), "eosq_scores launch")) return EOSQ_ERR_CUDA;
     return EOSQ_OK;
@@ -416,7 +436,7 @@ extern "C" int eosq_encode_host(eosq_ctx *ctx, const void *host_blocks, int in_d
     int rc = check_shape(n, d, bits);
     if (rc != EOSQ_OK) return rc;
     if (num_blocks == 0) return EOSQ_OK;
-    if (!host_blocks || !cache_required_ok(host_out) || !arena || (reinterpret_cast<uintptr_t>(arena) & 255u))
+    if (!host_blocks || !cache_required_ok(host_out) || !arena || (reinterpret_cast<uintptr_t>(arena) & 255u) || !on_ctx_device(ctx))
         return EOSQ_ERR_INVALID_ARG;
     if (arena_bytes < eosq_encode_host_arena_bytes(num_blocks, n, d, bits, in_dtype)) return EOSQ_ERR_BUFFER_TOO_SMALL;
     if (!host_path_ready(ctx)) return EOSQ_ERR_CUDA;
@@ -484,7 +504,7 @@ extern "C" int eosq_encode_host(eosq_ctx *ctx, const void *host_blocks, int in_d
 
 extern "C" int eosq_check_status(eosq_ctx *ctx, const int32_t *status, int64_t num_blocks, int64_t *flagged,
                                  void *cuda_stream) {
-    if (!ctx || num_blocks < 0 || (num_blocks > 0 && !status)) return EOSQ_ERR_INVALID_ARG;
+    if (!ctx || num_blocks < 0 || (num_blocks > 0 && !status) || !on_ctx_device(ctx)) return EOSQ_ERR_INVALID_ARG;
     std::vector<int32_t> h(static_cast<size_t>(num_blocks));
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     if (num_blocks > 0) {

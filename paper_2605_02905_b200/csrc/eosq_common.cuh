@@ -56,6 +56,11 @@ constexpr int64_t CHUNK_BLOCKS = 1184;  // 8 per SM on 148 SMs: what the second 
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Raises a kernel's dynamic shared-memory limit, once per kernel and device (the attribute belongs
+// to the device's copy of the function, so a second GPU in the same process needs its own call).
+// Implemented in eosq_api.cu.
+bool ensure_dynamic_smem(const void *kernel, size_t bytes);
+
 // Carve the scratch arrays of one chunk (capacity `cap` blocks) out of `base`; returns the bytes
 // used.  With base = nullptr only the size is computed.
 inline size_t carve(void *base, int64_t cap, Workspace *ws) {
@@ -83,7 +88,7 @@ inline size_t carve(void *base, int64_t cap, Workspace *ws) {
 
 }  // namespace eosq
 
-enum Stage { ST_GRAM = 0, ST_TRIDIAG_A, ST_TRIDIAG_B, ST_TRIDIAG_C, ST_EIGVALS, ST_SPECTRAL, ST_QUANT, ST_DECODE, ST_SCORES, ST_REDO, ST_OTHER };
+enum Stage { ST_GRAM = 0, ST_TRIDIAG_A, ST_TRIDIAG_B, ST_EIGVALS, ST_SPECTRAL, ST_QUANT, ST_DECODE, ST_SCORES, ST_REDO, ST_OTHER };
 
 struct eosq_ctx {
     struct Timed {
@@ -148,16 +153,11 @@ void launch_quant_plain(const void *blocks, int in_dtype, int64_t nb, int n, con
 // Same outputs from the tensor cores (fp16 blocks only); `out` is already offset to the chunk.
 bool launch_quant_tc(const void *blocks_all, int64_t block0, int64_t nb, int n, const Workspace &ws, const Rotation &rot,
                      const Codebook &cb, const eosq_cache_t &out, int *err, int sm_count, cudaStream_t s);
-void launch_decode_plain(const eosq_cache_t &cache, int64_t nb, int n, const Rotation &rot, const Codebook &cb,
-                         void *out_blocks, int out_dtype, cudaStream_t s);
 bool decode_tc_supported(const eosq_cache_t &cache, int bits, const void *out_blocks);
 bool launch_decode_tc(const eosq_cache_t &cache, int64_t nb, int n, const Rotation &rot, const Codebook &cb, void *out_blocks,
                       int out_dtype, int *err, int sm_count, cudaStream_t s);
-void launch_scores_plain(const eosq_cache_t &cache, int64_t heads, int64_t bph, int64_t head_stride, int n,
-                         const Rotation &rot, const Codebook &cb, const __half *q, int G, float scale,
-                         float *scores, cudaStream_t s);
-
-// Tensor-core version of the logits (2-bit codes); returns false if nothing was enqueued.
+// Attention logits on the tensor cores; `supported` checks the 16-byte alignment the kernel's bulk copies
+// need, the launcher returns false if nothing was enqueued.
 bool scores_tc_supported(const eosq_cache_t &cache, int bits, int n);
 bool launch_scores_tc(const eosq_cache_t &cache, int64_t heads, int64_t bph, int64_t head_stride, int n, const Rotation &rot,
                       const Codebook &cb, const __half *q, int G, float scale, float *scores, int *err, int sm_count,

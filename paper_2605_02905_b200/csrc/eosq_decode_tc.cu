@@ -313,12 +313,7 @@ bool decode_tc_supported(const eosq_cache_t &cache, int bits, const void *out_bl
 
 template <typename Tout, int BITS>
 static bool launch_decode_tc_as(const DecodeArgs &a, const CUtensorMap &omap, int grid, cudaStream_t s) {
-    static bool configured = false;
-    if (!configured) {
-        if (cudaFuncSetAttribute(decode_tc_kernel<Tout, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(DT_SMEM)) != cudaSuccess)
-            return false;
-        configured = true;
-    }
+    if (!ensure_dynamic_smem(reinterpret_cast<const void *>(decode_tc_kernel<Tout, BITS>), DT_SMEM)) return false;
     decode_tc_kernel<Tout, BITS><<<grid, DT_THREADS, DT_SMEM, s>>>(a, omap);
     return true;
 }

@@ -520,21 +520,10 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
     }
 }
 
-bool scores_ws_supported(const eosq_cache_t &cache, int bits, int n) {
-    auto aligned = [](const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; };
-    return bits >= 1 && bits <= 4 && n >= 128 && (n % 8) == 0 && aligned(cache.codes) && aligned(cache.norms) && aligned(cache.P) && aligned(cache.V);
-}
-
 template <int BITS>
 static bool launch_scores_ws_as(WsArgs &a, int G, int grid, const CUtensorMap &m4, const CUtensorMap &m8, const CUtensorMap &m12,
                                 const float *pi_t, uint8_t *wimg, int64_t *kernels, cudaStream_t s) {
-    static bool configured = false;
-    if (!configured) {
-        if (cudaFuncSetAttribute(scores_ws_kernel<BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(WsLayout<BITS>::SMEM_BYTES)) != cudaSuccess)
-            return false;
-        configured = true;
-    }
+    if (!ensure_dynamic_smem(reinterpret_cast<const void *>(scores_ws_kernel<BITS>), WsLayout<BITS>::SMEM_BYTES)) return false;
     for (int g0 = 0; g0 < G; g0 += WS_NQ) {
         a.g0 = g0;
         scores_w_kernel<<<a.heads, D, 0, s>>>(pi_t, a.q, G, g0, wimg);

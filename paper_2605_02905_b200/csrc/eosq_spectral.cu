@@ -561,7 +561,7 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
         // the sums over the whole spectrum have a pole at z, so they are taken at six points
         // z + m h, m = -3 .. 3 without 0, the known eigenvalues are subtracted there, and what is left
         // (smooth: the tail lies well below z) is interpolated to z, exact for polynomials of degree 5.
-        // h = z / 64, or less when a neighbouring known eigenvalue is closer than 3.5 h.
+        // h = z / 64, or a little less when a known eigenvalue would sit on a sample point.
         // Warps 1 .. 3 take these sums and Step 3 while warp 0 factorises for the eigenvectors below.
         if (warp > 0) {
             const int e = tid - 32;
@@ -569,9 +569,22 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
                 const int i = e / 6, m6 = e % 6;
                 const int mm = (m6 < 3) ? m6 - 3 : m6 - 2;   // -3, -2, -1, 1, 2, 3
                 const double z = lam[i];
-                double gnn = z - lam[i + 1];
-                if (i > 0) gnn = fmin(gnn, lam[i - 1] - z);
-                const double h = fmin(z * (1.0 / 64.0), gnn * (1.0 / 3.5));
+                // A known eigenvalue right at a sample point would be subtracted with a large
+                // cancellation error: shrink h until every other known eigenvalue keeps a quarter
+                // step away from all six points (the six threads of a vector find the same h).
+                double h = z * (1.0 / 64.0);
+#pragma unroll 1
+                for (int attempt = 0; attempt < 8; ++attempt) {
+                    double nearest = 1e300;
+#pragma unroll 1
+                    for (int j = 0; j < EV_TOP; ++j) {
+                        if (j == i) continue;
+                        const double t = fabs(lam[j] - z) / h;   // in steps
+                        if (t < 3.5) nearest = fmin(nearest, fabs(t - rint(t)) + ((t < 0.5) ? 1.0 : 0.0));
+                    }
+                    if (nearest >= 0.25) break;
+                    h *= 0.8125;
+                }
                 const double x = fma(static_cast<double>(mm), h, z);
                 const double is = sp_rcp(mscale);
                 double f1, f2;
@@ -588,7 +601,6 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
                 const double w = (am == 1) ? 15.0 / 20.0 : ((am == 2) ? -6.0 / 20.0 : 1.0 / 20.0);
                 st1[e] = w * f1;
                 st2[e] = w * f2;
-                if (!(h > z * (1.0 / 16384.0))) atomicOr(&s_flags, EOSQ_BLOCK_CLUSTERED);
             }
             asm volatile("bar.sync 1, 96;" ::: "memory");
             // Step 3: Stieltjes transforms of F_e at z = lambda_i, D-transform, Eq. 9, Eq. 6.
@@ -838,12 +850,7 @@ void launch_eigvals(int64_t nb, const Workspace &ws, const int *list, const int 
 
 void launch_spectral(int64_t nb, int n, const Workspace &ws, const eosq_cache_t &out, int64_t block0, bool full,
                      cudaStream_t s) {
-    static bool configured = false;
-    if (!configured) {
-        cudaFuncSetAttribute(spectral_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             static_cast<int>(SPECTRAL_DYN_SMEM));
-        configured = true;
-    }
+    ensure_dynamic_smem(reinterpret_cast<const void *>(spectral_kernel), SPECTRAL_DYN_SMEM);
     spectral_kernel<<<static_cast<unsigned>(nb), SP_THREADS, SPECTRAL_DYN_SMEM, s>>>(n, ws, out, static_cast<long long>(block0), full);
 }
 

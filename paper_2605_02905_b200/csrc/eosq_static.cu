@@ -67,6 +67,10 @@ extern "C" int eosq_encode_static(eosq_ctx *ctx, const void *blocks, int in_dtyp
     int dev = -1;
     if (fail(ctx, cudaGetDevice(&dev), "cudaGetDevice")) return EOSQ_ERR_CUDA;
     if (dev < 0 || dev >= MAX_DEVICES) return EOSQ_ERR_UNSUPPORTED;
+    if (dev != ctx->device) {   // the context's error word and constants live on its own device
+        ctx->last_error = "the current CUDA device is not the one this context was created on";
+        return EOSQ_ERR_INVALID_ARG;
+    }
     std::lock_guard<std::mutex> lock(g_mu);
     PerDevice &pd = g_dev[dev];
     if (!pd.base) {

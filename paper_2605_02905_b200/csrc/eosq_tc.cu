@@ -233,12 +233,7 @@ __global__ void __launch_bounds__(GRAM_THREADS, 1) gram_tc_kernel(const __grid_c
 
 bool launch_gram_tc(const void *blocks_all, int64_t nb_all, int64_t block0, int64_t nb, int n, double *gram, int *err,
                     int sm_count, cudaStream_t s) {
-    static bool configured = false;
-    if (!configured) {
-        if (cudaFuncSetAttribute(gram_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(GRAM_SMEM)) != cudaSuccess)
-            return false;
-        configured = true;
-    }
+    if (!ensure_dynamic_smem(reinterpret_cast<const void *>(gram_tc_kernel), GRAM_SMEM)) return false;
     (void)nb_all;
     CUtensorMap tmap;
     const char *base = static_cast<const char *>(blocks_all) + static_cast<size_t>(block0) * n * D * 2;
@@ -564,12 +559,7 @@ __global__ void __launch_bounds__(QT_THREADS, 2) quant_tc_kernel(const __grid_co
 template <int BITS>
 static bool launch_quant_tc_bits(const CUtensorMap &tmap, int nb, int n, const Workspace &ws, const Rotation &rot,
                                  const Codebook &cb, const eosq_cache_t &out, int *err, int grid, cudaStream_t s) {
-    static bool configured = false;
-    if (!configured) {
-        if (cudaFuncSetAttribute(quant_tc_kernel<BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(QT_SMEM)) != cudaSuccess)
-            return false;
-        configured = true;
-    }
+    if (!ensure_dynamic_smem(reinterpret_cast<const void *>(quant_tc_kernel<BITS>), QT_SMEM)) return false;
     quant_tc_kernel<BITS><<<grid, QT_THREADS, QT_SMEM, s>>>(tmap, nb, n, ws, rot.pi, rot.pi_t, cb, out, err);
     return true;
 }

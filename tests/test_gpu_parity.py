@@ -290,3 +290,135 @@ def test_full_size_cache_sampled_blocks(ctx, bits, full):
     assert eosq.eosq_check_status(ctx, cache) == 0
     assert torch.all(torch.isfinite(dec[::257].float()))
     parity.compare_decode(sub_cache, dec[pick], bits, SEED, tol=1e-3)
+
+
+def _stratified(planted, is_key, want):
+    """Indices of blocks covering the planted ranks in `want` for keys and values (first match each)."""
+    pick = []
+    for key in (True, False):
+        for lo, hi in want:
+            hits = [i for i in range(len(planted)) if bool(is_key[i]) == key and lo <= planted[i] <= hi and i not in pick]
+            if hits:
+                pick.append(hits[0])
+    return sorted(pick)
+
+
+def test_ministral_shaped_blocks_rank_above_pilot_and_pure_noise(ctx):
+    """Config 3 (Ministral-8B shape, n = 1024): planted ranks up to 32, above the pilot k = 11, where the
+    single-pass rank test of Algorithm 2 inflates its own bulk edge and the selected rank collapses; 5 % of
+    the blocks are pure noise (rank 0).  Keys and values, sampled by planted rank; then the logits of
+    G = 16 queries per KV head (4 query heads x batch 4) against the compressed keys of the first head."""
+    w = synth.ministral_64k(max_blocks=136)            # head 0: K blocks 0..63, V blocks 64..127, then head 1's K
+    planted = w.planted_rank
+    pick = _stratified(planted, w.is_key, [(0, 0), (1, 4), (5, 11), (12, 20), (21, 32)])
+    assert any(planted[i] == 0 for i in pick) and any(planted[i] > 11 for i in pick)
+    dev, cache = _encode(ctx, w.blocks, 2, full=False)
+    flagged = {i: int(v) for i, v in enumerate(cache.status.cpu().tolist()) if v}
+    assert not flagged, flagged
+    rep, enc = parity.compare_encode(w.blocks, cache, 2, SEED, blocks_idx=pick)
+    rep["planted_vs_selected"] = [(int(planted[i]), int(cache.rank[i])) for i in pick]
+    _report("ministral_n1024", rep)
+    assert rep["e2e_out_band_fraction"] < 1e-4
+    sel = cache.rank.cpu().numpy()
+    # pure-noise value blocks must come out with rank 0 (key blocks still carry their outlier channels)
+    assert sel.max() <= 11 and all(sel[i] == 0 for i in range(len(planted)) if planted[i] == 0 and not w.is_key[i])
+    dec = eosq.eosq_decode(ctx, cache, SEED)
+    parity.compare_decode(cache, dec, 2, SEED, blocks_idx=pick[:3])
+    heads, bph, G = 1, 64, 16
+    q = synth.queries(heads, G, seed=12).cuda()
+    s = eosq.eosq_scores(ctx, cache, q, heads, bph, 2 * bph, SEED)
+    torch.cuda.synchronize()
+    worst = parity.compare_scores(cache, q, s, heads, bph, 2 * bph, 2, SEED, 1.0 / math.sqrt(128),
+                                  pairs=[(0, 0), (0, 17), (0, 63)])
+    print(f"\n[parity] ministral scores G=16: worst relative {worst:.3e}")
+
+
+@pytest.mark.parametrize("n", [256, 512, 1024, 2048, 4096])
+def test_sweep_points_around_the_detection_threshold(ctx, n):
+    """Config 4 (sweep): four spikes at {5, 1.5, 1.05, 0.9} x the BBP threshold, block lengths 256 .. 4096, every
+    code width.  The 0.9 x and 1.05 x spikes sit at the bulk edge and must not be kept; the 1.5 x one lands
+    close to the d^(-1/3) margin of the rank test."""
+    w = synth.kv_cache_blocks(f"sweep_n{n}", layers=1, kv_heads=1, tokens=3 * n, n=n, fixed_theta=[5.0, 1.5, 1.05, 0.9], seed=4)
+    pick = [0, 4] if n >= 2048 else [0, 2, 4]          # K blocks 0..2, V blocks 3..5
+    enc2 = None
+    hist = {}
+    for bits in (2, 1, 3, 4):
+        dev, cache = _encode(ctx, w.blocks, bits, full=(bits == 3))
+        rep, enc = parity.compare_encode(w.blocks, cache, bits, SEED, blocks_idx=pick)
+        if bits == 2:
+            enc2 = enc
+            for r in cache.rank.cpu().tolist():
+                hist[r] = hist.get(r, 0) + 1
+            rep["rank_histogram"] = hist
+            rep["min_margin"] = float(enc["margin"].min())
+        _report(f"sweep_n{n}_b{bits}", rep)
+        assert rep["e2e_out_band_fraction"] < 1e-4
+        # value blocks: the 5 x spike always kept, the 1.5 x one at most, the edge spikes never; key blocks
+        # add their four outlier channels
+        sel = cache.rank.cpu().numpy()
+        assert all(1 <= sel[i] <= 2 for i in range(len(sel)) if not w.is_key[i]), sel
+        assert all(1 <= sel[i] <= 6 for i in range(len(sel)) if w.is_key[i]), sel
+    dec = eosq.eosq_decode(ctx, cache, SEED)
+    parity.compare_decode(cache, dec, 4, SEED, blocks_idx=pick[:1])
+    assert enc2 is not None
+
+
+def test_block_at_the_rank_threshold_is_compared_separately(ctx):
+    """A block whose leading eigenvalue sits within 1e-4 of the rank cut (strength found by bisection on the
+    oracle): either side of the cut is a valid answer there, so the comparison must take its
+    near-threshold branch -- same rank and full parity, or a flagged mismatch -- and count the block."""
+    n, d = 256, 128
+    g = torch.Generator().manual_seed(11)
+    Z = torch.randn(n, d, generator=g, dtype=torch.float64) / math.sqrt(n)
+    u = torch.linalg.qr(torch.randn(n, 1, generator=g, dtype=torch.float64))[0]
+    v = torch.linalg.qr(torch.randn(d, 1, generator=g, dtype=torch.float64))[0]
+
+    def block(theta):
+        return ((Z + theta * (u @ v.T)) * 4.0).to(torch.float16)
+
+    def state(theta):
+        S = block(theta).double().numpy()
+        sig = oracle.svd(S)[0]
+        sp = oracle.eoptshrink_spectrum(n, d, sig)
+        return sp["rank"], sp["margin"]
+
+    lo, hi = 0.5, 3.0
+    assert state(lo)[0] == 0 and state(hi)[0] == 1
+    theta = hi
+    for _ in range(60):
+        mid = 0.5 * (lo + hi)
+        r, margin = state(mid)
+        theta = mid
+        if margin < 5e-5:
+            break
+        if r == 0:
+            lo = mid
+        else:
+            hi = mid
+    r, margin = state(theta)
+    assert margin < parity.RANK_MARGIN, margin
+    blocks = torch.stack([block(theta), block(theta * 1.5)])
+    dev, cache = _encode(ctx, blocks, 2, full=False)
+    rep, enc = parity.compare_encode(blocks, cache, 2, SEED)
+    rep["margin"] = margin
+    _report("near_threshold", rep)
+    assert rep["near_threshold_blocks"] == 1
+    assert int(cache.rank[1]) == 1 and int(cache.rank[0]) in (0, 1)
+
+
+def test_unaligned_cache_arrays_are_rejected(ctx):
+    """Decode and scores move the cache with 16-byte bulk copies: a misaligned array is an argument error."""
+    L = eosq.lib()
+    blocks = torch.randn(2, 256, 128, generator=torch.Generator().manual_seed(2)).to(torch.float16)
+    dev, cache = _encode(ctx, blocks, 2)
+    st = cache.struct()
+    st.codes = cache.codes.data_ptr() + 4
+    stream = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    out = torch.empty((2, 256, 128), dtype=torch.float32, device="cuda")
+    rc = L.eosq_decode(ctx._h, ctypes.addressof(st), 2, 256, 128, 2, ctypes.c_uint64(SEED), out.data_ptr(), eosq.EOSQ_F32, stream)
+    assert rc == eosq.EOSQ_ERR_INVALID_ARG
+    q = synth.queries(1, 4, seed=1).cuda()
+    s = torch.empty((1, 4, 512), dtype=torch.float32, device="cuda")
+    rc = L.eosq_scores(ctx._h, ctypes.addressof(st), 1, 2, 2, 256, 128, 2, ctypes.c_uint64(SEED), q.data_ptr(), 4,
+                       ctypes.c_float(0.1), s.data_ptr(), stream)
+    assert rc == eosq.EOSQ_ERR_INVALID_ARG
