@@ -5,6 +5,8 @@
 // All arithmetic here is double precision: the bulk eigenvalues sit two to three orders of
 // magnitude below the largest outlier, and the rank test and the shrunk values must agree with a
 // double-precision reference to 1e-4 relative or better.
+#include <algorithm>
+
 #include "eosq_common.cuh"
 
 namespace eosq {
@@ -30,10 +32,11 @@ constexpr int EV_PE_INVALID = -(1 << 28);   // exponent marking a p_d whose magn
 constexpr int EV_GROUP = 8;               // recurrence steps between two range checks
 constexpr int EV_PAD = EV_GROUP;          // entries past the end that the look-ahead may read
 
+template <bool COUNT>
 __device__ __forceinline__ void sturm_step(const double2 de, double x, double &p0, double &p1, unsigned &cnt) {
     const double t = de.y * p0;
     const double p2 = fma(de.x - x, p1, -t);
-    cnt += static_cast<unsigned>(__double2hiint(p1) ^ __double2hiint(p2)) >> 31;
+    if (COUNT) cnt += static_cast<unsigned>(__double2hiint(p1) ^ __double2hiint(p2)) >> 31;
     p0 = p1;
     p1 = p2;
 }
@@ -43,6 +46,8 @@ __device__ __forceinline__ void sturm_step(const double2 de, double x, double &p
 // of the next group are fetched before the current group's chain of dependent multiply-adds
 // starts, and the pair is brought back to within 2^+-300 of one after every group: eight steps
 // move it by at most 2^13 upwards and, even with full cancellation in every step, 2^-424 downwards.
+// Without COUNT only p_d(x) is worked out (its sign is all a bracket around a single eigenvalue needs).
+template <bool COUNT = true>
 __device__ __forceinline__ int sturm_eval(const double2 *__restrict__ sde, double x, double &pm, int &pe) {
     double p0 = 1.0, p1 = sde[0].x - x;
     unsigned cnt = static_cast<unsigned>(__double2hiint(p1)) >> 31;
@@ -57,7 +62,7 @@ __device__ __forceinline__ int sturm_eval(const double2 *__restrict__ sde, doubl
 #pragma unroll
         for (int i = 0; i < EV_GROUP; ++i) nxt[i] = q[i];
 #pragma unroll
-        for (int i = 0; i < EV_GROUP; ++i) sturm_step(cur[i], x, p0, p1, cnt);
+        for (int i = 0; i < EV_GROUP; ++i) sturm_step<COUNT>(cur[i], x, p0, p1, cnt);
         const int e0 = (__double2hiint(p0) >> 20) & 0x7ff, e1 = (__double2hiint(p1) >> 20) & 0x7ff;
         const int em = max(e0, e1);
         if (static_cast<unsigned>(em - 723) > 600u) {
@@ -76,18 +81,20 @@ __device__ __forceinline__ int sturm_eval(const double2 *__restrict__ sde, doubl
         for (int i = 0; i < EV_GROUP; ++i) cur[i] = nxt[i];
     }
 #pragma unroll
-    for (int i = 0; i < (D - 1) - NG * EV_GROUP; ++i) sturm_step(cur[i], x, p0, p1, cnt);
+    for (int i = 0; i < (D - 1) - NG * EV_GROUP; ++i) sturm_step<COUNT>(cur[i], x, p0, p1, cnt);
     pm = p1;
     pe = esum;
     return static_cast<int>(cnt);
 }
 
-// Which eigenvalues a call resolves.  Algorithm 2 reads individually only lambda_1 .. lambda_{2k+r+1}
-// (Steps 1 and 2; r <= k, so 3k + 1 = 34 of them at d = 128); the rest of the spectrum enters
-// through sums that the spectral kernel takes from the characteristic polynomial.  The smallest
-// eigenvalue is resolved as well: it decides whether the tensor-core Gram matrix was accurate
-// enough.  With FULL every eigenvalue is resolved (the optional `eig` output).
-constexpr int EV_TOP = 3 * KPILOT + 1;
+// Which eigenvalues are resolved.  Algorithm 2 reads individually only lambda_1 .. lambda_{k+r+1} and
+// lambda_{2k+1}, lambda_{2k+r+1} (Steps 1 and 2; r <= k); the rest of the spectrum enters through sums
+// that the spectral kernel takes from the characteristic polynomial.  The fast kernel resolves the
+// EV_EXPL = 32 largest (one lane each) and, for the rare ranks 10 and 11, lambda_{2k+r+1} (index 32 or
+// 33) in a second round; the full kernel resolves every eigenvalue (the optional `eig` output).
+constexpr int EV_EXPL = 32;
+constexpr int EV_TOP = 3 * KPILOT + 1;   // entries of lam the spectral kernel may read without the full spectrum
+static_assert(2 * KPILOT + 9 < EV_EXPL && EV_TOP <= EV_EXPL + 2, "ranks up to 9 find lambda_{2k+r+1} among the first 32");
 
 // With `mark_list` set (first pass over tensor-core Gram matrices), a block whose smallest
 // eigenvalue is not at least REDO_RATIO of the largest (this includes non-finite spectra) is queued
@@ -280,6 +287,185 @@ __global__ void __launch_bounds__(FULL ? D : 64) eigvals_kernel(const double *__
         eigvals_block<FULL>(diag, off, lam, list ? list[li] : li, mark_list, mark_count);
         if (!list) break;
         __syncthreads();   // the shared state is reused by the next listed block
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// The fast eigenvalue kernel: one warp per block, lane t resolves lambda_{t+1}.  Same method as
+// above (first pass on a geometric grid, here of 64 points; bisection on Sturm counts; regula falsi
+// on p_d once a bracket holds one eigenvalue), with two savings: while every lane of the warp
+// interpolates, the evaluations skip the sign counting (the sign of p_d tells the side), and nothing
+// beyond the 32 largest eigenvalues is resolved unless the rank turns out to be 10 or 11.
+// ------------------------------------------------------------------------------------------
+constexpr int EVT_WARPS = 4;     // blocks per CTA
+constexpr int EVT_GRID = 64;     // points of the first pass
+
+struct EvtShared {
+    double2 sde[D + EV_PAD];
+    double pm[EVT_GRID];
+    int cnt[EVT_GRID], pe[EVT_GRID];
+};
+
+// Shrinks the bracket of the eigenvalue with ascending index `target` (lanes with active = false only
+// keep the warp's evaluations company) and returns the polished root, in the scaled units of sde.
+__device__ __forceinline__ double evt_refine(const EvtShared &sh, int target, bool active, double glo, double ghi, bool geometric) {
+    auto point = [&](int t) -> double {
+        if (t < 0) return glo;
+        if (geometric) return ghi * exp2(-(9.0 * 3.321928094887362 / (EVT_GRID - 1)) * static_cast<double>(EVT_GRID - 1 - t));
+        return glo + (ghi - glo) * static_cast<double>(t + 1) / static_cast<double>(EVT_GRID);
+    };
+    int t = -1;                      // largest grid index with count <= target
+#pragma unroll
+    for (int step = EVT_GRID / 2; step > 0; step >>= 1)
+        if (t + step < EVT_GRID && sh.cnt[t + step] <= target) t += step;
+    double lo = point(t), hi = (t + 1 < EVT_GRID) ? point(t + 1) : ghi;
+    if (t == EVT_GRID - 1) lo = hi;
+    int clo = (t >= 0) ? sh.cnt[t] : 0, chi = (t + 1 < EVT_GRID) ? sh.cnt[t + 1] : D;
+    double flo = (t >= 0) ? sh.pm[t] : 0.0, fhi = (t + 1 < EVT_GRID) ? sh.pm[t + 1] : 0.0;
+    double tlo = flo, thi = fhi;
+    int elo = (t >= 0) ? sh.pe[t] : EV_PE_INVALID, ehi = (t + 1 < EVT_GRID) ? sh.pe[t + 1] : EV_PE_INVALID;
+    int replaced = 0, poor = 0;
+    for (int it = 0; it < EV_MAX_ITER; ++it) {
+        const double mid = 0.5 * (lo + hi);
+        const bool done = !active || (hi - lo) <= fmax(2e-15, 1e-8 * fabs(mid));
+        if (__all_sync(0xffffffffu, done)) break;
+        double x = mid;
+        const bool single = chi - clo == 1 && elo > EV_PE_INVALID / 2 && ehi > EV_PE_INVALID / 2 && tlo != 0.0 && thi != 0.0;
+        if (single && poor < 3 && (hi - lo) <= EV_SECANT_WIDTH * fabs(mid)) {
+            const double r = scalbn(fhi / flo, max(-2000, min(2000, ehi - elo)));   // p_d(hi) / p_d(lo), negative
+            if (r < 0.0) {
+                const double xs = lo + (hi - lo) / (1.0 - r);
+                if (xs > lo && xs < hi) x = xs;
+            }
+        }
+        const bool secant = x != mid;
+        const double width = hi - lo;
+        double pmv;
+        int pev, c;
+        // a lane that is done or holds a single eigenvalue with both end values can do without the count
+        if (__all_sync(0xffffffffu, done || single)) {
+            sturm_eval<false>(sh.sde, x, pmv, pev);
+            const bool same_as_lo = (__double2hiint(pmv) < 0) == (__double2hiint(tlo) < 0);
+            c = (pev > EV_PE_INVALID / 2 && pmv != 0.0) ? (same_as_lo ? clo : chi) : chi;
+            if (!(pev > EV_PE_INVALID / 2 && pmv != 0.0)) c = sturm_eval<true>(sh.sde, x, pmv, pev);   // the value was lost: count after all
+        } else {
+            c = sturm_eval<true>(sh.sde, x, pmv, pev);
+        }
+        if (c > target) {
+            hi = x;
+            chi = c;
+            fhi = pmv;
+            thi = pmv;
+            ehi = pev;
+            if (secant && replaced > 0) flo *= 0.5;
+            replaced = 1;
+        } else {
+            lo = x;
+            clo = c;
+            flo = pmv;
+            tlo = pmv;
+            elo = pev;
+            if (secant && replaced < 0) fhi *= 0.5;
+            replaced = -1;
+        }
+        poor = (hi - lo > 0.5 * width) ? poor + 1 : 0;
+    }
+    double xr = 0.5 * (lo + hi);
+    if (chi - clo == 1 && elo > EV_PE_INVALID / 2 && ehi > EV_PE_INVALID / 2 && tlo != 0.0) {
+        const double r = scalbn(thi / tlo, max(-2000, min(2000, ehi - elo)));
+        if (r < 0.0) {
+            const double xs = lo + (hi - lo) / (1.0 - r);
+            if (xs >= lo && xs <= hi) xr = xs;
+        }
+    }
+    return xr;
+}
+
+__global__ void __launch_bounds__(32 * EVT_WARPS) eigvals_top_kernel(const double *__restrict__ diag, const double *__restrict__ off,
+                                                                     double *__restrict__ lam, int nb, const int *__restrict__ list,
+                                                                     const int *__restrict__ count, int *__restrict__ mark_list,
+                                                                     int *__restrict__ mark_count) {
+    __shared__ __align__(16) EvtShared shs[EVT_WARPS];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    EvtShared &sh = shs[warp];
+    const int total = list ? *count : nb;
+    for (int li = blockIdx.x * EVT_WARPS + warp; li < total; li += gridDim.x * EVT_WARPS) {
+        const int blk = list ? list[li] : li;
+        const size_t base = static_cast<size_t>(blk) * D;
+        double dv[4], ev[4], m = 0.0;
+        bool nonfinite = false;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int i = lane + 32 * q;
+            dv[q] = diag[base + i];
+            ev[q] = (i < D - 1) ? off[base + i] : 0.0;
+            m = fmax(m, fmax(fabs(dv[q]), fabs(ev[q])));
+            nonfinite |= !(fabs(dv[q]) < 1e300) || !(fabs(ev[q]) < 1e300);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = fmax(m, __shfl_xor_sync(0xffffffffu, m, o));
+        if (__any_sync(0xffffffffu, nonfinite) || m == 0.0) {
+            // a non-finite entry poisons the whole spectrum (NaN, and a second pass if there is one); a zero matrix has a zero spectrum
+            const bool bad = m != 0.0;
+            lam[base + lane] = bad ? nan("") : 0.0;
+            if (lane < 2) lam[base + EV_EXPL + lane] = bad ? nan("") : 0.0;
+            if (bad && mark_list && lane == 0) mark_list[atomicAdd(mark_count, 1)] = blk;
+            continue;
+        }
+        const double scale = 1.0 / m;
+        __syncwarp();   // the previous block's last reads of sde are over
+        double glo = 1e300, ghi = -1e300;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int i = lane + 32 * q;
+            const double sd = dv[q] * scale, se = fabs(ev[q] * scale);
+            double se_prev = __shfl_up_sync(0xffffffffu, se, 1);
+            if (lane == 0) se_prev = (q > 0) ? fabs(off[base + i - 1] * scale) : 0.0;
+            sh.sde[i] = make_double2(sd, (i > 0) ? fmax(se_prev * se_prev, EV_E2_FLOOR) : 0.0);
+            glo = fmin(glo, sd - se - se_prev);
+            ghi = fmax(ghi, sd + se + se_prev);
+        }
+        if (lane < EV_PAD) sh.sde[D + lane] = make_double2(0.0, 0.0);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            glo = fmin(glo, __shfl_xor_sync(0xffffffffu, glo, o));
+            ghi = fmax(ghi, __shfl_xor_sync(0xffffffffu, ghi, o));
+        }
+        glo -= 1e-10 * (fabs(glo) + 1.0);
+        ghi += 1e-10 * (fabs(ghi) + 1.0);
+        __syncwarp();
+        const bool geometric = ghi > 0.0;
+#pragma unroll 1
+        for (int q = 0; q < EVT_GRID / 32; ++q) {
+            const int t = lane + 32 * q;
+            const double x = geometric ? ghi * exp2(-(9.0 * 3.321928094887362 / (EVT_GRID - 1)) * static_cast<double>(EVT_GRID - 1 - t))
+                                       : glo + (ghi - glo) * static_cast<double>(t + 1) / static_cast<double>(EVT_GRID);
+            double pmv;
+            int pev;
+            sh.cnt[t] = sturm_eval<true>(sh.sde, x, pmv, pev);
+            sh.pm[t] = pmv;
+            sh.pe[t] = pev;
+        }
+        __syncwarp();
+        const double xs = evt_refine(sh, D - 1 - lane, true, glo, ghi, geometric);
+        lam[base + lane] = xs * m;
+        // Is the smallest eigenvalue below REDO_RATIO of the largest?  One count tells.
+        const double x_top = __shfl_sync(0xffffffffu, xs, 0);
+        if (mark_list) {
+            double pmv;
+            int pev;
+            const int below = sturm_eval<true>(sh.sde, REDO_RATIO * x_top, pmv, pev);
+            if (lane == 0 && (below > 0 || !(x_top > 0.0))) mark_list[atomicAdd(mark_count, 1)] = blk;
+        }
+        // Ranks 10 and 11 make Step 2 read lambda_{2k+r+1}, index 32 or 33: resolve both then.
+        const double edge_c = 1.0 / (cbrt(4.0) - 1.0);
+        const double l_k = __shfl_sync(0xffffffffu, xs, KPILOT), l_2k = __shfl_sync(0xffffffffu, xs, 2 * KPILOT);
+        const double lam_plus = l_k + edge_c * (l_k - l_2k);
+        const unsigned passing = __ballot_sync(0xffffffffu, lane <= KPILOT && (xs / lam_plus - 1.0 > 1.0 / cbrt(static_cast<double>(D))));
+        if (__popc(passing) >= 10) {
+            const double x2 = evt_refine(sh, D - 1 - (EV_EXPL + (lane & 1)), lane < 2, glo, ghi, geometric);
+            if (lane < 2) lam[base + EV_EXPL + lane] = x2 * m;
+        }
     }
 }
 
@@ -502,7 +688,7 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
     const size_t base = static_cast<size_t>(b) * D;
     {
         // lam[EV_TOP .. D-2] holds eigenvalues only when the full spectrum was asked for
-        lam[tid] = (full || tid < EV_TOP || tid == D - 1) ? ws.lam[base + tid] : 0.0;
+        lam[tid] = (full || tid < EV_TOP) ? ws.lam[base + tid] : 0.0;   // (indices 32, 33: only meaningful, and only read, for ranks 10, 11)
         dd[tid] = ws.diag[base + tid];
         ee[tid] = ws.off[base + tid];
         tt[tid] = ws.tau[base + tid];
@@ -523,7 +709,7 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
     const double edge_c = 1.0 / (cbrt(4.0) - 1.0);
     const double cut = 1.0 / cbrt(static_cast<double>(D));
     const double lam_plus = lam[KPILOT] + edge_c * (lam[KPILOT] - lam[2 * KPILOT]);
-    const bool pass = (tid < EV_TOP) && (lam[tid] / lam_plus - 1.0 > cut);
+    const bool pass = (tid <= KPILOT) && (lam[tid] / lam_plus - 1.0 > cut);
     int rank = __syncthreads_count(pass);
     if (tid == 0) {
         unsigned f = 0u;
@@ -535,10 +721,10 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
 
     if (rank > 0) {
         // Step 2: k imputed atoms behind the outliers; the observed eigenvalues after them are known
-        // one by one up to lambda_EV_TOP, the rest (the tail) only through sums.
+        // one by one up to lambda_EV_EXPL, the rest (the tail) only through sums.
         {
             double a = 0.0;
-            if (tid >= rank + KPILOT && tid < EV_TOP) a = lam[tid];
+            if (tid >= rank + KPILOT && tid < EV_EXPL) a = lam[tid];
             else if (tid >= rank && tid < rank + KPILOT) {
                 const int jj = tid - rank + 1;
                 const double bs = lam[KPILOT + rank];
@@ -557,7 +743,7 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
             sde[tid] = make_double2(dd[tid] * is, (tid > 0) ? fmax(se * se, EV_E2_FLOOR) : 0.0);
         }
         __syncthreads();
-        // Tail sums  sum_{j > EV_TOP} 1 / (lambda_j - z)  and  sum 1 / (lambda_j - z)^2  at z = lambda_i:
+        // Tail sums  sum_{j > EV_EXPL} 1 / (lambda_j - z)  and  sum 1 / (lambda_j - z)^2  at z = lambda_i:
         // the sums over the whole spectrum have a pole at z, so they are taken at six points
         // z + m h, m = -3 .. 3 without 0, the known eigenvalues are subtracted there, and what is left
         // (smooth: the tail lies well below z) is interpolated to z, exact for polynomials of degree 5.
@@ -577,7 +763,7 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
                 for (int attempt = 0; attempt < 8; ++attempt) {
                     double nearest = 1e300;
 #pragma unroll 1
-                    for (int j = 0; j < EV_TOP; ++j) {
+                    for (int j = 0; j < EV_EXPL; ++j) {
                         if (j == i) continue;
                         const double t = fabs(lam[j] - z) / h;   // in steps
                         if (t < 3.5) nearest = fmin(nearest, fabs(t - rint(t)) + ((t < 0.5) ? 1.0 : 0.0));
@@ -592,7 +778,7 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
                 f1 *= is;
                 f2 *= is * is;
 #pragma unroll 2
-                for (int j = 0; j < EV_TOP; ++j) {
+                for (int j = 0; j < EV_EXPL; ++j) {
                     const double inv = sp_rcp(lam[j] - x);
                     f1 -= inv;
                     f2 = fma(-inv, inv, f2);
@@ -607,7 +793,7 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
             for (int i = warp - 1; i < rank; i += SP_WARPS - 1) {
                 const double z = lam[i];
                 double ms = 0.0, msp = 0.0;
-                for (int j = rank + lane; j < EV_TOP; j += 32) {
+                for (int j = rank + lane; j < EV_EXPL; j += 32) {
                     const double inv = sp_rcp(atoms[j] - z);
                     ms += inv;
                     msp = fma(inv, inv, msp);
@@ -844,8 +1030,13 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
 }
 
 void launch_eigvals(int64_t nb, const Workspace &ws, const int *list, const int *count, int *mark_list, bool full, cudaStream_t s) {
-    if (full) eigvals_kernel<true><<<list_grid(nb, list), D, 0, s>>>(ws.diag, ws.off, ws.lam, list, count, mark_list, ws.redo_count);
-    else eigvals_kernel<false><<<list_grid(nb, list), 64, 0, s>>>(ws.diag, ws.off, ws.lam, list, count, mark_list, ws.redo_count);
+    if (full) {
+        eigvals_kernel<true><<<list_grid(nb, list), D, 0, s>>>(ws.diag, ws.off, ws.lam, list, count, mark_list, ws.redo_count);
+    } else {
+        const int64_t work = list ? std::min<int64_t>(nb, LIST_GRID) : nb;
+        const unsigned grid = static_cast<unsigned>(std::max<int64_t>(1, (work + EVT_WARPS - 1) / EVT_WARPS));
+        eigvals_top_kernel<<<grid, 32 * EVT_WARPS, 0, s>>>(ws.diag, ws.off, ws.lam, static_cast<int>(nb), list, count, mark_list, ws.redo_count);
+    }
 }
 
 void launch_spectral(int64_t nb, int n, const Workspace &ws, const eosq_cache_t &out, int64_t block0, bool full,

@@ -153,20 +153,27 @@ def test_two_bit_decode_with_a_ragged_last_tile(ctx, n):
 
 
 def test_many_blocks_cross_the_chunk_boundary_and_are_deterministic(ctx):
-    """More blocks than one internal chunk: every block must equal its stand-alone encoding."""
-    w = synth.kv_cache_blocks("chunks", layers=2, kv_heads=3, tokens=128 * 102, n=128, rank_hi=4, seed=50)
-    assert w.blocks.shape[0] == 1224
-    dev, cache = _encode(ctx, w.blocks, 2)
-    dev2, cache2 = _encode(ctx, w.blocks, 2)
+    """More blocks than one internal chunk (18944): every block must equal its stand-alone encoding."""
+    w = synth.kv_cache_blocks("chunks", layers=2, kv_heads=3, tokens=128 * 1580, n=128, rank_hi=4, seed=50, device="cuda")
+    B = w.blocks.shape[0]
+    assert B == 18960
+    cache = eosq.eosq_encode(ctx, w.blocks, 2, SEED)
+    cache2 = eosq.eosq_encode(ctx, w.blocks, 2, SEED)
+    torch.cuda.synchronize()
     for name in ("codes", "norms", "rank", "sigma", "phi", "V", "status", "eig"):
         assert torch.equal(getattr(cache, name), getattr(cache2, name)), name
-    pick = [0, 591, 592, 611, 1183, 1184, 1223]
+    del cache2
+    pick = [0, 591, 18943, 18944, B - 1]
     for b in pick:
-        _, single = _encode(ctx, w.blocks[b:b + 1], 2)
+        single = eosq.eosq_encode(ctx, w.blocks[b:b + 1].contiguous(), 2, SEED)
         assert torch.equal(single.codes[0], cache.codes[b]) and torch.equal(single.norms[0], cache.norms[b])
         r = int(single.rank[0])
         assert r == int(cache.rank[b]) and torch.equal(single.P[0, :r], cache.P[b, :r])
-    rep, enc = parity.compare_encode(w.blocks, cache, 2, SEED, blocks_idx=pick)
+    sub = w.blocks[pick].cpu()
+    sub_cache = eosq.Cache.allocate(len(pick), w.n, w.d, 2)
+    for name in ("codes", "norms", "rank", "sigma", "phi", "P", "V", "status", "eig", "lambda_plus", "vr32", "coef"):
+        getattr(sub_cache, name).copy_(getattr(cache, name)[pick])
+    rep, enc = parity.compare_encode(sub, sub_cache, 2, SEED)
     _report("chunks", rep)
 
 
