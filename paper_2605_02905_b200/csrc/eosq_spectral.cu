@@ -542,7 +542,6 @@ __device__ __forceinline__ void charpoly_sums(const double2 *__restrict__ sde, d
 constexpr int SP_THREADS = 128, SP_WARPS = SP_THREADS / 32;
 constexpr int LU_LANES = 12;
 static_assert(KPILOT < LU_LANES && KPILOT <= 3 * SP_WARPS, "one LU column and one warp slot per kept vector");
-constexpr size_t SPECTRAL_DYN_SMEM = sizeof(double) * 4 * D * LU_LANES;
 
 // Back-transformation x = H_0 H_1 ... H_{D-3} y of the kept vectors, normalisation, and the stores of
 // the right singular vectors.  The reflectors (rows of R, 1 KB each) are staged through shared memory
@@ -551,8 +550,10 @@ constexpr size_t SPECTRAL_DYN_SMEM = sizeof(double) * 4 * D * LU_LANES;
 // lane: rows 16 m + 2 sub, + 1), so a dot product needs three shuffle stages and four vectors share
 // every instruction.  Reflector k is zero up to index k, and whole 16-row chunks of zeros are skipped.
 constexpr int BT_ROWS = 16;                 // reflector rows per stage
+// dynamic shared memory: the vectors, then the two factor arrays or (later) the two reflector stages
+constexpr size_t SPECTRAL_DYN_SMEM = sizeof(double) * (D * LU_LANES + (2 * BT_ROWS * D > 2 * D * LU_LANES ? 2 * BT_ROWS * D : 2 * D * LU_LANES));
 constexpr int BT_BAR_FULL = 2, BT_BAR_EMPTY = 4;   // named barriers: + stage
-static_assert(2 * BT_ROWS * D <= 3 * D * LU_LANES, "the ring reuses the storage of the factorisations");
+
 
 // (barrier numbers are spelled out: a number in a register makes the compiler reserve all sixteen)
 __device__ __forceinline__ void bt_bar_sync(int id) {
@@ -670,17 +671,16 @@ __device__ __forceinline__ void sp_back_transform(const double *__restrict__ R, 
 
 __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspace ws, eosq_cache_t out, long long block0, bool full) {
     __shared__ double lam[D], dd[D], ee[D], tt[D], atoms[D];
-    __shared__ double inv_e[D];              // reciprocals of the (clamped) subdiagonal entries
     __shared__ __align__(16) double2 sde[D];  // (d_i, e_{i-1}^2) of the scaled matrix, for the characteristic polynomial
     __shared__ double st1[6 * KPILOT], st2[6 * KPILOT];   // weighted samples of the tail sums around each kept eigenvalue
     __shared__ double s_max[SP_WARPS];
     __shared__ double s_phi[RMAX], s_sig[RMAX];
     __shared__ unsigned s_flags;
     extern __shared__ double dyn[];
-    double *lu_l = dyn;                      // multipliers                      [D][12]
-    double *lu_d = dyn + D * LU_LANES;       // reciprocal pivots                [D][12]
-    double *lu_u = dyn + 2 * D * LU_LANES;   // first superdiagonal of U         [D][12]
-    double *yv = dyn + 3 * D * LU_LANES;     // iteration vectors                [D][12]
+    double *yv = dyn;                        // D+, then the vectors             [D][12]
+    double *lu_l = dyn + D * LU_LANES;       // e_i / D+_i                       [D][12]
+    double *lu_u = dyn + 2 * D * LU_LANES;   // e_i / D-_{i+1}                   [D][12]
+    double *ring = dyn + D * LU_LANES;       // the back-transformation's reflector stages take the place of lu_l, lu_u
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = blockIdx.x;
@@ -734,10 +734,7 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
             atoms[tid] = a;
         }
         const double floor_piv = 1.2e-16 * fmax(fabs(lam[0]), 1e-300);
-        {   // pivots taken from the subdiagonal do not depend on the vector: their reciprocals are shared
-            double l = ee[tid];
-            if (!(fabs(l) >= floor_piv)) l = (l < 0.0) ? -floor_piv : floor_piv;
-            inv_e[tid] = sp_rcp(l);
+        {
             const double is = (mscale > 0.0) ? 1.0 / mscale : 0.0;
             const double se = (tid > 0) ? fabs(ee[tid - 1] * is) : 0.0;
             sde[tid] = make_double2(dd[tid] * is, (tid > 0) ? fmax(se * se, EV_E2_FLOOR) : 0.0);
@@ -832,165 +829,61 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
             }
         }
 
-        // Kept eigenvectors of the tridiagonal matrix: (T - mu I) = P L U with partial pivoting,
-        // two steps of inverse iteration (the kept eigenvalues are separated from their
-        // neighbours by far more than their error, so each step gains many digits).  Lane i of
-        // warp 0 owns vector i (column i of the arrays).  The iterate is left unnormalised: it can
-        // grow by at most 1 / floor_piv per step, and the back-transformation normalises at the end.
+        // Kept eigenvectors of the tridiagonal matrix from its twisted factorisation: with the
+        // pivots of T - mu I = L+ D+ L+^T taken from the top,  D+_{i+1} = (d_{i+1} - mu) - e_i^2 / D+_i,
+        // and of U- D- U-^T taken from the bottom,  D-_i = (d_i - mu) - e_i^2 / D-_{i+1},
+        // gamma_i = D+_i + D-_i - (d_i - mu) is the residual of the vector z that starts with z_r = 1
+        // at index r and runs  z_i = -(e_i / D+_i) z_{i+1}  upwards and  z_{i+1} = -(e_i / D-_{i+1}) z_i
+        // downwards: (T - mu I) z = gamma_r e_r.  r = argmin |gamma| gives a residual of the order of
+        // the error of mu, which is at rounding level here, so one such vector is as good as inverse
+        // iteration converged.  Lane i of warp 0 owns vector i (column i of the arrays).
         if (warp == 0 && lane < rank) {
-            // A lone warp pays the full latency of every instruction, so these loops are written for
-            // few instructions per row: selects instead of branches, pointers that advance by
-            // constants, the pivot bits of 32 rows in one register.
             const int c = lane;
             const double mu = lam[c];
-            unsigned piv[4];
-            double d_i = dd[0] - mu, u_i = ee[0];
-            {
-                double *pl = lu_l + c, *pd = lu_d + c, *pu = lu_u + c;
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    unsigned word = 0u;
-#pragma unroll 1
-                    for (int ii = 0; ii < 32; ii += 4) {
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const int i = 32 * q + ii + j;
-                            if (i < D - 1) {
-                                const double l = ee[i];
-                                const double d_next = dd[i + 1] - mu;
-                                const double u_next = ee[i + 1];   // ee[D - 1] is zero
-                                // the reciprocal of the diagonal candidate starts before the pivot choice is known
-                                const double ds = (fabs(d_i) >= floor_piv) ? d_i : ((d_i < 0.0) ? -floor_piv : floor_piv);
-                                const double inv_d = sp_rcp(ds);
-                                const bool keep = fabs(d_i) >= fabs(l);
-                                // keep: row i stays.  Otherwise rows i and i + 1 change places and U gets a
-                                // second superdiagonal entry, e_{i+1}.
-                                const double inv = keep ? inv_d : inv_e[i];   // serves the elimination and the back substitution
-                                const double fact = (keep ? l : d_i) * inv;
-                                const double uu = keep ? u_i : d_next, other = keep ? d_next : u_i;
-                                pl[j * LU_LANES] = fact;
-                                pd[j * LU_LANES] = inv;
-                                pu[j * LU_LANES] = uu * inv;   // U's superdiagonal over its pivot
-                                d_i = fma(-fact, uu, other);
-                                u_i = keep ? u_next : -fact * u_next;
-                                word |= (keep ? 0u : 1u) << j;
-                            }
-                        }
-                        word = (word << 28) | (word >> 4);   // rotate: after eight groups bit r belongs to row 32 q + r
-                        pl += 4 * LU_LANES;
-                        pd += 4 * LU_LANES;
-                        pu += 4 * LU_LANES;
-                    }
-                    piv[q] = word;
+            // forward pivots; yv keeps D+ until the vector takes its place
+            double dp = dd[0] - mu;
+#pragma unroll 4
+            for (int i = 0; i < D - 1; ++i) {
+                if (!(fabs(dp) >= floor_piv)) dp = (dp < 0.0) ? -floor_piv : floor_piv;
+                const double e = ee[i];
+                const double lp = e * sp_rcp(dp);
+                yv[i * LU_LANES + c] = dp;
+                lu_l[i * LU_LANES + c] = lp;
+                dp = fma(-lp, e, dd[i + 1] - mu);
+            }
+            yv[(D - 1) * LU_LANES + c] = dp;
+            // backward pivots, and the twist index on the way
+            double dm = dd[D - 1] - mu;
+            double gbest = fabs(dp);   // gamma_{D-1} = D+_{D-1} (D-_{D-1} is d - mu itself)
+            int rbest = D - 1;
+#pragma unroll 4
+            for (int i = D - 2; i >= 0; --i) {
+                if (!(fabs(dm) >= floor_piv)) dm = (dm < 0.0) ? -floor_piv : floor_piv;
+                const double e = ee[i];
+                const double um = e * sp_rcp(dm);
+                lu_u[i * LU_LANES + c] = um;
+                const double t = dd[i] - mu;
+                dm = fma(-um, e, t);
+                const double gam = fabs(yv[i * LU_LANES + c] + dm - t);
+                if (gam < gbest) {
+                    gbest = gam;
+                    rbest = i;
                 }
             }
-            if (!(fabs(d_i) >= floor_piv)) d_i = (d_i < 0.0) ? -floor_piv : floor_piv;
-            lu_d[(D - 1) * LU_LANES + c] = 1.0 / d_i;
-            lu_u[(D - 1) * LU_LANES + c] = 0.0;
-            for (int i = 0; i < D; ++i) {
-                const double f = (i + 1) * 0.6180339887498949;
-                yv[i * LU_LANES + c] = 0.5 + (f - floor(f));
+            // the vector, left unnormalised (the back-transformation normalises at the end)
+            double ss = 1.0;
+            yv[rbest * LU_LANES + c] = 1.0;
+            double z = 1.0;
+            for (int i = rbest - 1; i >= 0; --i) {
+                z = -lu_l[i * LU_LANES + c] * z;
+                yv[i * LU_LANES + c] = z;
+                ss = fma(z, z, ss);
             }
-            double ss = 0.0;
-            for (int it = 0; it < 2; ++it) {
-                // forward: apply the row interchanges and L^-1.  Entries are fetched a group of four
-                // ahead (the stores of a group never reach the entries already fetched).
-                double carry = yv[c];
-                {
-                    double *py = yv + c;
-                    const double *pl = lu_l + c;
-                    double ny[4], nl[4];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        ny[j] = py[(1 + j) * LU_LANES];
-                        nl[j] = pl[j * LU_LANES];
-                    }
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        unsigned word = piv[q];
-#pragma unroll 1
-                        for (int ii = 0; ii < 32; ii += 4) {
-                            double cy[4], cl[4];
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                cy[j] = ny[j];
-                                cl[j] = nl[j];
-                                if (32 * q + ii + 4 + j < D - 1) {   // false only in the very last group
-                                    ny[j] = py[(5 + j) * LU_LANES];
-                                    nl[j] = pl[(4 + j) * LU_LANES];
-                                }
-                            }
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                if (32 * q + ii + j < D - 1) {
-                                    const bool swap = (word >> j) & 1u;
-                                    const double a = swap ? cy[j] : carry, other = swap ? carry : cy[j];
-                                    py[j * LU_LANES] = a;
-                                    carry = fma(-cl[j], a, other);
-                                }
-                            }
-                            word >>= 4;
-                            py += 4 * LU_LANES;
-                            pl += 4 * LU_LANES;
-                        }
-                    }
-                }
-                // backward: U^-1, as x_i = a_i - b_i x_{i+1} - c_i x_{i+2} with the coefficients
-                // prepared off the chain, so that one multiply-add separates consecutive entries.
-                // Rows go down from D - 2 in groups of four, row 32 q + ii + 3 - j in slot j.
-                double x1 = carry * lu_d[(D - 1) * LU_LANES + c];
-                yv[(D - 1) * LU_LANES + c] = x1;
-                double x2 = 0.0;
-                ss = x1 * x1;
-                {
-                    double *py = yv + (D - 4) * LU_LANES + c;   // row 32 q + ii of the current group
-                    const double *pd = lu_d + (D - 4) * LU_LANES + c, *pu = lu_u + (D - 4) * LU_LANES + c;
-                    const double *pe = ee + (D - 4) + 1;         // pe[r] = e_{i+1} for row i = 32 q + ii + r
-                    double ny[4], nd[4], nb[4], ne[4];
-#pragma unroll
-                    for (int j = 1; j < 4; ++j) {   // slot 0 of the first group would be row D - 1
-                        ny[j] = py[(3 - j) * LU_LANES];
-                        nd[j] = pd[(3 - j) * LU_LANES];
-                        nb[j] = pu[(3 - j) * LU_LANES];
-                        ne[j] = pe[3 - j];
-                    }
-                    ny[0] = nd[0] = nb[0] = ne[0] = 0.0;
-#pragma unroll
-                    for (int q = 3; q >= 0; --q) {
-                        const unsigned word = piv[q];
-#pragma unroll 1
-                        for (int ii = 28; ii >= 0; ii -= 4) {
-                            const unsigned bits = word >> ii;
-                            double ca[4], cb[4], cc[4];
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                ca[j] = ny[j] * nd[j];
-                                cb[j] = nb[j];
-                                cc[j] = ((bits >> (3 - j)) & 1u) ? ne[j] * nd[j] : 0.0;
-                                if (32 * q + ii >= 4) {   // false only in the very last group
-                                    ny[j] = py[(-1 - j) * LU_LANES];
-                                    nd[j] = pd[(-1 - j) * LU_LANES];
-                                    nb[j] = pu[(-1 - j) * LU_LANES];
-                                    ne[j] = pe[-1 - j];
-                                }
-                            }
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                if (32 * q + ii + 3 - j <= D - 2) {
-                                    const double x = fma(-cb[j], x1, fma(-cc[j], x2, ca[j]));
-                                    py[(3 - j) * LU_LANES] = x;
-                                    ss = fma(x, x, ss);
-                                    x2 = x1;
-                                    x1 = x;
-                                }
-                            }
-                            py -= 4 * LU_LANES;
-                            pd -= 4 * LU_LANES;
-                            pu -= 4 * LU_LANES;
-                            pe -= 4;
-                        }
-                    }
-                }
+            z = 1.0;
+            for (int i = rbest; i < D - 1; ++i) {
+                z = -lu_u[i * LU_LANES + c] * z;
+                yv[(i + 1) * LU_LANES + c] = z;
+                ss = fma(z, z, ss);
             }
             if (!(ss > 0.0 && ss < 1e300)) atomicOr(&s_flags, EOSQ_BLOCK_NOT_CONVERGED);
         }
@@ -1001,7 +894,7 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
     // are no longer needed after the barrier above).
     const double *R = ws.gram + static_cast<size_t>(b) * D * D;
     float *vr = ws.vr + static_cast<size_t>(b) * RMAX * D;
-    if (rank > 0) sp_back_transform(R, tt, yv, dyn, rank, warp, lane, vr, out, gb);
+    if (rank > 0) sp_back_transform(R, tt, yv, ring, rank, warp, lane, vr, out, gb);
     // rows >= rank of V are zero; scalars
     for (int e = tid; e < RMAX * D; e += SP_THREADS) {
         if (e / D >= rank) {
