@@ -107,18 +107,23 @@ template <int G>
 struct TtShared {
     double xu[2][G * TT_PSTRIDE];   // published row x (zero up to its own index), permuted
     double pp[2][G * TT_PSTRIDE];   // p, permuted (zero for finished indices)
-    double sspart[2][G];            // partial sums of squares of x[k+2..], one per publishing thread
+    double scal[2][4];              // per parity of k: beta_k, gamma_k, 2K_k (the first two from the publisher of row k)
     double wsum[2][8];              // per-warp parts of u . A u
     double dg[8 * G], of[8 * G], ta[8 * G];
 };
 
-// The G threads that hold row r (row slot AR = r / G of their tiles) publish x = A[r][r+1..] into
-// buffer `nxt`.  With UPDATE the pending rank-2 update of step r - 1 (vectors in buffer nxt ^ 1,
-// u_{r-1}[r] = uown, (p - 2K u)[r] = sown) is applied to the row first; the stored row is left as
-// it is, the next sweep brings it up to date like every other row.  Tensor-memory loads are
-// warp-wide instructions, so the whole warp of the holders runs this and `mine` marks the holders.
+// The G threads that hold row r (row slot AR = r / G of their tiles) turn it into reflector r and
+// publish that: x = A[r][r+1..], beta = -sign(x_{r+1}) ||x||, gamma = 1 / (beta (beta - x_{r+1})),
+// u = x - beta e_{r+1} into buffer `nxt` (zero up to index r), beta and gamma into scal[nxt], the
+// tridiagonal entries d_r, beta into dg / of / ta, and u into row r of the matrix in global memory
+// (`grow`).  With UPDATE the pending rank-2 update of step r - 1 (vectors in buffer nxt ^ 1,
+// u_{r-1}[r] = uown, (p - 2K u)[r] = sown) is applied to the row first; the stored row is left as it
+// is, the next sweep brings it up to date like every other row.  Tensor-memory loads and shuffles
+// are warp-wide, so the whole warp of the holders runs this and `mine` marks the holders (they are
+// G consecutive lanes).
 template <int G, int AR, bool UPDATE>
-__device__ __forceinline__ void tt_publish(uint32_t tb, int r, int nxt, int tc, bool mine, TtShared<G> &sh, double uown, double sown) {
+__device__ __forceinline__ void tt_publish(uint32_t tb, int r, int nxt, int lane, int tc, bool mine, TtShared<G> &sh, double uown,
+                                           double sown, double *__restrict__ grow) {
     uint32_t raw[16];
     tmem_ld16(tb + 16u * AR, raw);
     double uj[8], pj[8];
@@ -144,52 +149,20 @@ __device__ __forceinline__ void tt_publish(uint32_t tb, int r, int nxt, int tc, 
         }
         const int col = tc + G * b;
         double t = tt_get(raw, b);
-        if (UPDATE) {
-            // u_{r-1} at index r is x - beta, which is uown; right of it the raw x is u
-            const double ujf = (b == AR && col == r) ? uown : uj[b];
-            t = fma(-uown, pj[b], fma(-sown, ujf, t));
-        }
+        if (UPDATE) t = fma(-uown, pj[b], fma(-sown, uj[b], t));
         if (b == AR && mine && col == r) sh.dg[r] = t;
         x[b] = (col > r) ? t : 0.0;
         const double s = (col > r + 1) ? t : 0.0;
         if (b & 1) ss1 = fma(s, s, ss1);
         else ss0 = fma(s, s, ss0);
     }
-    if (mine) {
-        double2 *dst = reinterpret_cast<double2 *>(&sh.xu[nxt][tc * TT_PSTRIDE]);
+    // ||x[r+2..]||^2 over the holders, x_{r+1} from the holder of that column
+    double ss = ss0 + ss1;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) dst[q] = make_double2(x[2 * q], x[2 * q + 1]);
-        sh.sspart[nxt][tc] = ss0 + ss1;
-    }
-}
-
-// One step k of a team, with (k + 1) / G == K0.  `grow` is the global row that receives the
-// reflector; t is the thread's index within its team.  twoK of the pending update comes in, that
-// of this step goes out.
-template <int G, int K0, int TEAMS>
-__device__ __forceinline__ void tt_step(uint32_t tb, int k, int kend, int t, int team, TtShared<G> &sh, double *__restrict__ grow,
-                                        double &twoK_prev) {
-    constexpr int N = 8 * G, TEAM_THREADS = G * G, NW = TEAM_THREADS / 32;
-    const int lane = t & 31, warp = t >> 5, tr = t / G, tc = t & (G - 1);
-    tt_sync<TEAMS, TEAM_THREADS>(team);
-    const int cur = k & 1, prv = cur ^ 1;
-    // reflector scalars from the published row
-    double ss;
-    {
-        const double2 *sp = reinterpret_cast<const double2 *>(sh.sspart[cur]);
-        double part[G / 2];
-#pragma unroll
-        for (int q = 0; q < G / 2; ++q) {
-            const double2 v = sp[q];
-            part[q] = v.x + v.y;
-        }
-#pragma unroll
-        for (int w = G / 4; w >= 1; w >>= 1)
-#pragma unroll
-            for (int q = 0; q < w; ++q) part[q] = part[2 * q] + part[2 * q + 1];
-        ss = part[0];
-    }
-    const double alpha = sh.xu[cur][tt_pos<G>(k + 1)];
+    for (int o = G / 2; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    const bool next_slot = ((r + 1) / G) != AR;   // column r + 1 sits in column slot AR or AR + 1
+    const double xsel = next_slot ? x[(AR + 1) & 7] : x[AR];
+    const double alpha = __shfl_sync(0xffffffffu, xsel, (lane & ~(G - 1)) | ((r + 1) & (G - 1)));
     double beta = alpha, gamma = 0.0;
     if (ss > 0.0) {
         const double sq = fma(alpha, alpha, ss);
@@ -197,33 +170,61 @@ __device__ __forceinline__ void tt_step(uint32_t tb, int k, int kend, int t, int
         beta = (alpha >= 0.0) ? -nrm : nrm;
         gamma = tt_rcp(fma(fabs(alpha), nrm, sq));   // 1 / (beta (beta - alpha))
     }
-    if (t < N) grow[t] = (t > k) ? sh.xu[cur][tt_pos<G>(t)] - ((t == k + 1) ? beta : 0.0) : 0.0;
-    if (t == 0) {
-        sh.of[k] = beta;
-        sh.ta[k] = gamma;
+    if (tc == ((r + 1) & (G - 1))) {
+        if (next_slot) x[(AR + 1) & 7] -= beta;
+        else x[AR] -= beta;
     }
-    const bool col_holder = tc == ((k + 1) & (G - 1)), row_holder = tr == ((k + 1) & (G - 1));   // of index k + 1 (slot K0)
-    // column-side vectors: u of this step, u' and p' of the pending update
+    if (mine) {
+        double2 *dst = reinterpret_cast<double2 *>(&sh.xu[nxt][tc * TT_PSTRIDE]);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) dst[q] = make_double2(x[2 * q], x[2 * q + 1]);
+#pragma unroll
+        for (int b = 0; b < 8; ++b) grow[tc + G * b] = x[b];
+        if (tc == 0) {
+            sh.scal[nxt][0] = beta;
+            sh.scal[nxt][1] = gamma;
+            sh.of[r] = beta;
+            sh.ta[r] = gamma;
+        }
+    }
+}
+
+// One step k of a team, with (k + 1) / G == K0: the sweep with reflector k (published before the
+// first barrier, together with beta_k and gamma_k), p_k, and then, by the warp that holds row k + 1,
+// 2K_k and reflector k + 1.  `trow0` is row 0 of the matrix in global memory; t is the thread's index
+// within its team.
+template <int G, int K0, int TEAMS>
+__device__ __forceinline__ void tt_step(uint32_t tb, int k, int kend, int t, int team, TtShared<G> &sh, double *__restrict__ trow0) {
+    constexpr int TEAM_THREADS = G * G, NW = TEAM_THREADS / 32;
+    const int lane = t & 31, warp = t >> 5, tr = t / G, tc = t & (G - 1);
+    const int cur = k & 1, prv = cur ^ 1;
+    // What does not depend on reflector k is fetched while its publisher is still at work: the
+    // vectors u' and p' of the pending update (complete since the last barrier).
     double ujn[8], ujp[8], pjp[8];
     {
-        const double2 *un = reinterpret_cast<const double2 *>(&sh.xu[cur][tc * TT_PSTRIDE]);
         const double2 *up = reinterpret_cast<const double2 *>(&sh.xu[prv][tc * TT_PSTRIDE]);
         const double2 *pq = reinterpret_cast<const double2 *>(&sh.pp[prv][tc * TT_PSTRIDE]);
 #pragma unroll
         for (int q = K0 / 2; q < 4; ++q) {
-            const double2 a = un[q], b = up[q], c = pq[q];
-            ujn[2 * q] = a.x;
-            ujn[2 * q + 1] = a.y;
+            const double2 b = up[q], c = pq[q];
             ujp[2 * q] = b.x;
             ujp[2 * q + 1] = b.y;
             pjp[2 * q] = c.x;
             pjp[2 * q + 1] = c.y;
         }
-        if (col_holder) ujn[K0] -= beta;
     }
-    // The sweep: every live element is brought up to date, written back and used for A u.  The
-    // pending update needs no correction at index k (u' there is x' - beta'): row and column k are
-    // finished and nothing reads them again.
+    tt_sync<TEAMS, TEAM_THREADS>(team);
+    const double gamma = sh.scal[cur][1], twoK_prev = sh.scal[prv][2];   // 2K' comes from the publisher, like gamma
+    {
+        const double2 *un = reinterpret_cast<const double2 *>(&sh.xu[cur][tc * TT_PSTRIDE]);
+#pragma unroll
+        for (int q = K0 / 2; q < 4; ++q) {
+            const double2 a = un[q];
+            ujn[2 * q] = a.x;
+            ujn[2 * q + 1] = a.y;
+        }
+    }
+    // The sweep: every live element is brought up to date, written back and used for A u.
     double acc[8];
     const double *ur = &sh.xu[prv][tr * TT_PSTRIDE], *pr = &sh.pp[prv][tr * TT_PSTRIDE];
 #pragma unroll
@@ -253,16 +254,12 @@ __device__ __forceinline__ void tt_step(uint32_t tb, int k, int kend, int t, int
     double tloc = 0.0;
     {
         const double2 *un = reinterpret_cast<const double2 *>(&sh.xu[cur][tr * TT_PSTRIDE]);
-        double uin[8];
 #pragma unroll
         for (int q = K0 / 2; q < 4; ++q) {
             const double2 v = un[q];
-            uin[2 * q] = v.x;
-            uin[2 * q + 1] = v.y;
+            tloc = fma(v.x, acc[2 * q], tloc);
+            tloc = fma(v.y, acc[2 * q + 1], tloc);
         }
-        if (row_holder) uin[K0] -= beta;
-#pragma unroll
-        for (int a = K0; a < 8; ++a) tloc = fma(uin[a], acc[a], tloc);
     }
     const bool hA = tc & (G / 2), hB = tc & (G / 4), hC = tc & (G / 8);
     double v4[4], v2[2], v1;
@@ -288,31 +285,34 @@ __device__ __forceinline__ void tt_step(uint32_t tb, int k, int kend, int t, int
     if (lane == 0) sh.wsum[cur][warp] = tloc;
     tmem_st_wait();   // this thread's own stores; nobody else reads its lane
     tt_sync<TEAMS, TEAM_THREADS>(team);
-    double uAu;
-    {
-        const double2 *wp = reinterpret_cast<const double2 *>(&sh.wsum[cur][0]);
-        const double2 w0 = wp[0];
-        uAu = w0.x + w0.y;
-        if (NW == 8) {
-            const double2 w1 = wp[1], w2 = wp[2], w3 = wp[3];
-            uAu = (uAu + (w1.x + w1.y)) + ((w2.x + w2.y) + (w3.x + w3.y));
+    // The warp that holds row k + 1 (row slot K0 of G of its lanes) finishes the step: 2K from the
+    // warps' parts of u . A u, then the next reflector.
+    if (warp == (((k + 1) & (G - 1)) * G) / 32) {
+        double uAu;
+        {
+            const double2 *wp = reinterpret_cast<const double2 *>(&sh.wsum[cur][0]);
+            const double2 w0 = wp[0];
+            uAu = w0.x + w0.y;
+            if (NW == 8) {
+                const double2 w1 = wp[1], w2 = wp[2], w3 = wp[3];
+                uAu = (uAu + (w1.x + w1.y)) + ((w2.x + w2.y) + (w3.x + w3.y));
+            }
         }
-    }
-    const double twoK = gamma * gamma * uAu;
-    twoK_prev = twoK;
-    // the next reflector comes from row k + 1 (row slot K0 of its G holders, all in one warp)
-    if (k + 1 < kend && warp == (((k + 1) & (G - 1)) * G) / 32) {
-        const int p1 = tt_pos<G>(k + 1);
-        const double uown = sh.xu[cur][p1] - beta;
-        const double sown = fma(-twoK, uown, sh.pp[cur][p1]);
-        tt_publish<G, K0, true>(tb, k + 1, prv, tc, row_holder, sh, uown, sown);
+        const double twoK = gamma * gamma * uAu;
+        if (lane == 0) sh.scal[cur][2] = twoK;
+        if (k + 1 < kend) {
+            const int p1 = tt_pos<G>(k + 1);
+            const double uown = sh.xu[cur][p1];
+            const double sown = fma(-twoK, uown, sh.pp[cur][p1]);
+            tt_publish<G, K0, true>(tb, k + 1, prv, lane, tc, tr == ((k + 1) & (G - 1)), sh, uown, sown,
+                                    trow0 + static_cast<size_t>(k + 1) * D);
+        }
     }
 }
 
 template <int G, int K0, int LO, int HI, int TEAMS>
-__device__ __forceinline__ void tt_step_if(uint32_t tb, int k, int kend, int t, int team, TtShared<G> &sh, double *__restrict__ grow,
-                                           double &twoK_prev) {
-    if constexpr (K0 >= LO && K0 <= HI) tt_step<G, K0, TEAMS>(tb, k, kend, t, team, sh, grow, twoK_prev);
+__device__ __forceinline__ void tt_step_if(uint32_t tb, int k, int kend, int t, int team, TtShared<G> &sh, double *__restrict__ trow0) {
+    if constexpr (K0 >= LO && K0 <= HI) tt_step<G, K0, TEAMS>(tb, k, kend, t, team, sh, trow0);
 }
 
 // Steps [0, KE) of the reduction of the order-8G matrix whose element (i, j) sits at
@@ -364,6 +364,7 @@ __global__ void __launch_bounds__(G *G *TEAMS, MINB) tridiag_tm_kernel(double *_
             sh.pp[0][e] = 0.0;
             sh.pp[1][e] = 0.0;
         }
+        if (t < 8) sh.scal[t >> 2][t & 3] = 0.0;
         if constexpr (ORIGIN > 0) {   // the reflector rows of this range are full-width rows: zero left of the matrix
             for (int e = t; e < KE * (ORIGIN / 2); e += TEAM_THREADS) {
                 const int r = e / (ORIGIN / 2), c2 = e % (ORIGIN / 2);
@@ -372,21 +373,19 @@ __global__ void __launch_bounds__(G *G *TEAMS, MINB) tridiag_tm_kernel(double *_
         }
         tmem_st_wait();
         tt_sync<TEAMS, TEAM_THREADS>(team);
-        if ((t >> 5) == 0) tt_publish<G, 0, false>(tb, 0, 0, tc, tr == 0, sh, 0.0, 0.0);
-        double twoK_prev = 0.0;
+        if ((t >> 5) == 0) tt_publish<G, 0, false>(tb, 0, 0, t & 31, tc, tr == 0, sh, 0.0, 0.0, T);
         constexpr int HI = KE / G;
 #pragma unroll 1
         for (int k = 0; k < KE; ++k) {
-            double *grow = Gm + static_cast<size_t>(ORIGIN + k) * D + ORIGIN;
             switch ((k + 1) / G) {
-                case 0: tt_step_if<G, 0, 0, HI, TEAMS>(tb, k, KE, t, team, sh, grow, twoK_prev); break;
-                case 1: tt_step_if<G, 1, 0, HI, TEAMS>(tb, k, KE, t, team, sh, grow, twoK_prev); break;
-                case 2: tt_step_if<G, 2, 0, HI, TEAMS>(tb, k, KE, t, team, sh, grow, twoK_prev); break;
-                case 3: tt_step_if<G, 3, 0, HI, TEAMS>(tb, k, KE, t, team, sh, grow, twoK_prev); break;
-                case 4: tt_step_if<G, 4, 0, HI, TEAMS>(tb, k, KE, t, team, sh, grow, twoK_prev); break;
-                case 5: tt_step_if<G, 5, 0, HI, TEAMS>(tb, k, KE, t, team, sh, grow, twoK_prev); break;
-                case 6: tt_step_if<G, 6, 0, HI, TEAMS>(tb, k, KE, t, team, sh, grow, twoK_prev); break;
-                default: tt_step_if<G, 7, 0, HI, TEAMS>(tb, k, KE, t, team, sh, grow, twoK_prev); break;
+                case 0: tt_step_if<G, 0, 0, HI, TEAMS>(tb, k, KE, t, team, sh, T); break;
+                case 1: tt_step_if<G, 1, 0, HI, TEAMS>(tb, k, KE, t, team, sh, T); break;
+                case 2: tt_step_if<G, 2, 0, HI, TEAMS>(tb, k, KE, t, team, sh, T); break;
+                case 3: tt_step_if<G, 3, 0, HI, TEAMS>(tb, k, KE, t, team, sh, T); break;
+                case 4: tt_step_if<G, 4, 0, HI, TEAMS>(tb, k, KE, t, team, sh, T); break;
+                case 5: tt_step_if<G, 5, 0, HI, TEAMS>(tb, k, KE, t, team, sh, T); break;
+                case 6: tt_step_if<G, 6, 0, HI, TEAMS>(tb, k, KE, t, team, sh, T); break;
+                default: tt_step_if<G, 7, 0, HI, TEAMS>(tb, k, KE, t, team, sh, T); break;
             }
         }
         // The update of the last step is still pending: apply it to what is left of the matrix
@@ -394,19 +393,19 @@ __global__ void __launch_bounds__(G *G *TEAMS, MINB) tridiag_tm_kernel(double *_
         // at the very end, as the last diagonal and off-diagonal entries.
         {
             constexpr int AF = KE / G;
+            tt_sync<TEAMS, TEAM_THREADS>(team);   // 2K of the last step comes from another warp
             const int kl = KE - 1, cur = kl & 1;
-            const double beta = sh.of[kl];
+            const double twoK_prev = sh.scal[cur][2];
             double uj[8], pj[8];
 #pragma unroll
             for (int b = AF; b < 8; ++b) {
-                const int col = tc + G * b;
-                uj[b] = sh.xu[cur][tc * TT_PSTRIDE + b] - ((col == KE) ? beta : 0.0);
+                uj[b] = sh.xu[cur][tc * TT_PSTRIDE + b];
                 pj[b] = sh.pp[cur][tc * TT_PSTRIDE + b];
             }
 #pragma unroll
             for (int a = AF; a < 8; ++a) {
                 const int row = tr + G * a;
-                const double ui = sh.xu[cur][tr * TT_PSTRIDE + a] - ((row == KE) ? beta : 0.0);
+                const double ui = sh.xu[cur][tr * TT_PSTRIDE + a];
                 const double si = fma(-twoK_prev, ui, sh.pp[cur][tr * TT_PSTRIDE + a]);
                 uint32_t raw[16];
                 tmem_ld16(tb + 16u * a, raw);
