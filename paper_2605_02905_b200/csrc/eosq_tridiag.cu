@@ -213,6 +213,8 @@ __device__ __forceinline__ void tt_step(uint32_t tb, int k, int kend, int t, int
             pjp[2 * q + 1] = c.y;
         }
     }
+    uint32_t raw0[16];
+    tmem_ld16(tb + 16u * K0, raw0);   // the first live row slot of the tile, too
     tt_sync<TEAMS, TEAM_THREADS>(team);
     const double gamma = sh.scal[cur][1], twoK_prev = sh.scal[prv][2];   // 2K' comes from the publisher, like gamma
     {
@@ -232,7 +234,12 @@ __device__ __forceinline__ void tt_step(uint32_t tb, int k, int kend, int t, int
         acc[a] = 0.0;
         if (a < K0) continue;
         uint32_t raw[16];
-        tmem_ld16(tb + 16u * a, raw);
+        if (a == K0) {
+#pragma unroll
+            for (int e = 0; e < 16; ++e) raw[e] = raw0[e];
+        } else {
+            tmem_ld16(tb + 16u * a, raw);
+        }
         const double uip = ur[a];
         const double sip = fma(-twoK_prev, uip, pr[a]);
         tt_wait16(raw);
@@ -261,6 +268,8 @@ __device__ __forceinline__ void tt_step(uint32_t tb, int k, int kend, int t, int
             tloc = fma(v.y, acc[2 * q + 1], tloc);
         }
     }
+    // (the five butterfly stages of u . A u are interleaved with the tree by hand: both are chains of
+    // shuffles and additions, and neither depends on the other)
     const bool hA = tc & (G / 2), hB = tc & (G / 4), hC = tc & (G / 8);
     double v4[4], v2[2], v1;
 #pragma unroll
@@ -268,20 +277,24 @@ __device__ __forceinline__ void tt_step(uint32_t tb, int k, int kend, int t, int
         const double keep = hA ? acc[q + 4] : acc[q], send = hA ? acc[q] : acc[q + 4];
         v4[q] = keep + __shfl_xor_sync(0xffffffffu, send, G / 2);
     }
+    tloc += __shfl_xor_sync(0xffffffffu, tloc, 16);
 #pragma unroll
     for (int q = 0; q < 2; ++q) {
         const double keep = hB ? v4[q + 2] : v4[q], send = hB ? v4[q] : v4[q + 2];
         v2[q] = keep + __shfl_xor_sync(0xffffffffu, send, G / 4);
     }
+    tloc += __shfl_xor_sync(0xffffffffu, tloc, 8);
     {
         const double keep = hC ? v2[1] : v2[0], send = hC ? v2[0] : v2[1];
         v1 = keep + __shfl_xor_sync(0xffffffffu, send, G / 8);
     }
+    tloc += __shfl_xor_sync(0xffffffffu, tloc, 4);
     if (G == 16) v1 += __shfl_xor_sync(0xffffffffu, v1, 1);   // two threads per row are left: both get the sum
+    tloc += __shfl_xor_sync(0xffffffffu, tloc, 2);
     const int arow = (hA ? 4 : 0) + (hB ? 2 : 0) + (hC ? 1 : 0);
     const int irow = tr + G * arow;
     if (G == 8 || !(tc & 1)) sh.pp[cur][tt_pos<G>(irow)] = (irow > k) ? gamma * v1 : 0.0;
-    tloc = warp_sum(tloc);
+    tloc += __shfl_xor_sync(0xffffffffu, tloc, 1);
     if (lane == 0) sh.wsum[cur][warp] = tloc;
     tmem_st_wait();   // this thread's own stores; nobody else reads its lane
     tt_sync<TEAMS, TEAM_THREADS>(team);
