@@ -14,13 +14,14 @@
 // S is fp16 and exact as an operand; every other factor enters as a high and a low fp16 plane, so the
 // products carry about 2^-22 and the accumulation is fp32.
 //
-// One persistent CTA of 16 warps per SM:
+// One persistent CTA of 22 warps per SM:
 //   warp 0       TMA loads of the 128-token tiles into a ring of three stages
 //   warp 1       issues every MMA
-//   warps 4-7    per block: write V's rows of the operand, turn the W accumulator into the fix
+//   warps 2-5    per block: write V's rows of the operand, turn the W accumulator into the fix
 //                operand; per tile: turn P'' into the fix's A operand and store the left factors
 //                (one warp per quarter of the tensor-memory lanes)
-//   warps 8-15   epilogue: norm, thresholds scaled by the norm, codes, thread-local bit packing
+//   warps 6-21   epilogue, one token and 32 rotated coordinates per thread: norm, thresholds scaled
+//                by the norm, codes, thread-local bit packing
 // Two accumulator buffers let the MMAs of a tile run under the epilogue of the previous one.
 #include <algorithm>
 
@@ -36,7 +37,9 @@ bool make_block_tensor_map(const void *blocks, int64_t nb, int n, CUtensorMap *o
 namespace {
 
 constexpr int Q2_ERR_TIMEOUT = 2;        // same bit as the kernel this one replaced
-constexpr int Q2_THREADS = 512;
+constexpr int Q2_THREADS = 704;
+constexpr int Q2_EPI_WARPS = 16, Q2_EPI_FIRST = 6, Q2_CONV_FIRST = 2;
+constexpr int Q2_EPI_COLS = D / (Q2_EPI_WARPS / 4);   // 32 coordinates per epilogue thread
 constexpr int Q2_NST = 3;                // stages of the token-tile ring
 constexpr int Q2_NACC = 2;               // accumulator buffers
 constexpr int Q2_N = D + RMAX;           // 144 accumulator columns of the main product
@@ -82,13 +85,13 @@ __device__ __forceinline__ void q2_split8(const float (&m)[8], float scale, uint
     lo = make_uint4(l[0], l[1], l[2], l[3]);
 }
 
-// Barrier over the 256 epilogue threads that also tells every one of them whether any of them failed.
+// Barrier over the 512 epilogue threads that also tells every one of them whether any of them failed.
 __device__ __forceinline__ bool q2_epi_any(bool failed) {
     uint32_t r;
     asm volatile(
         "{\n\t.reg .pred p, q;\n\t"
         "setp.ne.u32 p, %1, 0;\n\t"
-        "bar.red.or.pred q, 1, 256, p;\n\t"
+        "bar.red.or.pred q, 1, 512, p;\n\t"
         "selp.u32 %0, 1, 0, q;\n\t}"
         : "=r"(r)
         : "r"(failed ? 1u : 0u)
@@ -103,7 +106,7 @@ __global__ void __launch_bounds__(Q2_THREADS, 1) quant_ws_kernel(const __grid_co
     extern __shared__ uint8_t q2_smem_raw[];
     __shared__ __align__(8) Q2Bars bars;
     __shared__ uint32_t tmem_base_s;
-    __shared__ float ss_part[Q2_NACC][2][128];
+    __shared__ float ss_part[Q2_NACC][4][128];
     __shared__ uint32_t fills[Q2_NST], drains[Q2_NST];   // loads issued / consumed per stage (for the clean-up after a failed wait)
     __shared__ volatile int abort_flag;
 
@@ -124,7 +127,7 @@ __global__ void __launch_bounds__(Q2_THREADS, 1) quant_ws_kernel(const __grid_co
             mbar_init(&bars.main_done[a], 1);
             mbar_init(&bars.a2_full[a], 4);
             mbar_init(&bars.y_full[a], 1);
-            mbar_init(&bars.acc_free[a], 8);
+            mbar_init(&bars.acc_free[a], Q2_EPI_WARPS);
         }
         mbar_init(&bars.v_free, 1);
         mbar_init(&bars.v_full, 4);
@@ -255,11 +258,11 @@ __global__ void __launch_bounds__(Q2_THREADS, 1) quant_ws_kernel(const __grid_co
                 }
             }
         }
-    } else if (warp >= 4 && warp < 8) {
+    } else if (warp >= Q2_CONV_FIRST && warp < Q2_CONV_FIRST + 4) {
         // ------------------------------------------------------------------ per-block operands, P'' -> fix operand, left factors
         const int q = warp & 3;                     // tensor-memory lanes [32 q, 32 q + 32) belong to this warp
         const int row = 32 * q + lane;              // a token of the tile, or a rotated coordinate c of W
-        const int st = tid - 128;                   // 0 .. 127 within the group
+        const int st = tid - 32 * Q2_CONV_FIRST;    // 0 .. 127 within the group
         const uint32_t lane_addr = tmem0 + (static_cast<uint32_t>(32 * q) << 16);
         uint32_t g = 0;
         bool ok = true;
@@ -369,9 +372,9 @@ __global__ void __launch_bounds__(Q2_THREADS, 1) quant_ws_kernel(const __grid_co
                 }
             }
         }
-    } else if (warp >= 8) {
-        // ------------------------------------------------------------------ epilogue: this thread owns token `row`, columns [64 h, 64 h + 64)
-        const int q = warp & 3, h = (warp >> 2) & 1;
+    } else if (warp >= Q2_EPI_FIRST) {
+        // ------------------------------------------------------------------ epilogue: this thread owns token `row`, coordinates [32 part, 32 part + 32)
+        const int q = warp & 3, part = (warp - Q2_EPI_FIRST) >> 2;
         const int row = 32 * q + lane;
         const uint32_t lane_addr = tmem0 + (static_cast<uint32_t>(32 * q) << 16);
         float thr[NTHR];
@@ -384,79 +387,86 @@ __global__ void __launch_bounds__(Q2_THREADS, 1) quant_ws_kernel(const __grid_co
             for (int t = 0; t < tiles; ++t, ++g) {
                 const int buf = g % Q2_NACC;
                 const bool got = mbar_wait(&bars.y_full[buf], (g / Q2_NACC) & 1u, &abort_flag);
-                float y[64];
-                float ss = 0.0f;
+                float y[Q2_EPI_COLS];
                 if (got) {
                     tc_fence_after_sync();
-                    uint32_t v0[32], v1[32];
-                    tmem_ld32(lane_addr + buf * Q2_ACC_COLS + 64u * h, v0);
-                    tmem_ld32(lane_addr + buf * Q2_ACC_COLS + 64u * h + 32u, v1);
+                    uint32_t v0[32];
+                    tmem_ld32(lane_addr + buf * Q2_ACC_COLS + static_cast<uint32_t>(Q2_EPI_COLS * part), v0);
                     tmem_ld_wait();
                     tc_fence_before_sync();
+                    float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f;
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) {
+                    for (int c = 0; c < Q2_EPI_COLS; c += 4) {
                         y[c] = __uint_as_float(v0[c]);
-                        y[32 + c] = __uint_as_float(v1[c]);
+                        y[c + 1] = __uint_as_float(v0[c + 1]);
+                        y[c + 2] = __uint_as_float(v0[c + 2]);
+                        y[c + 3] = __uint_as_float(v0[c + 3]);
+                        s0 = fmaf(y[c], y[c], s0);
+                        s1 = fmaf(y[c + 1], y[c + 1], s1);
+                        s2 = fmaf(y[c + 2], y[c + 2], s2);
+                        s3 = fmaf(y[c + 3], y[c + 3], s3);
                     }
-#pragma unroll
-                    for (int c = 0; c < 64; ++c) ss = fmaf(y[c], y[c], ss);
-                    ss_part[buf][h][row] = ss;
+                    ss_part[buf][part][row] = (s0 + s1) + (s2 + s3);
                 }
-                // both halves of every row are summed; every warp has read its part of the accumulator; and
-                // all 256 threads learn together whether one of them gave up waiting
+                // the four parts of every row are summed; every warp has read its part of the accumulator; and
+                // all epilogue threads learn together whether one of them gave up waiting
                 if (q2_epi_any(!got)) {
                     alive = false;
                     break;
                 }
                 if (lane == 0) mbar_arrive(&bars.acc_free[buf]);
-                const float tot = ss_part[buf][0][row] + ss_part[buf][1][row];
+                const float tot = (ss_part[buf][0][row] + ss_part[buf][1][row]) + (ss_part[buf][2][row] + ss_part[buf][3][row]);
                 const float rho = sqrtf(tot);
                 // thresholds scaled by the norm: y > thr rho decides as y / rho > thr does (a zero row keeps
                 // the plain thresholds, so that it gets the code of z = 0)
                 float ts[NTHR];
 #pragma unroll
                 for (int k = 0; k < NTHR; ++k) ts[k] = (rho > 0.0f) ? thr[k] * rho : thr[k];
-                unsigned long long wv[BITS];
+                // 32 codes of BITS bits: BITS words of 32 bits, coordinate j of the thread at bits [j BITS, (j+1) BITS)
+                uint32_t wv[BITS];
                 if (BITS == 3) {
+                    unsigned long long acc64 = 0ull;
+                    int filled = 0, wi = 0;
 #pragma unroll
-                    for (int k = 0; k < BITS; ++k) wv[k] = 0ull;
-#pragma unroll
-                    for (int c = 0; c < 64; ++c) {
+                    for (int c = 0; c < Q2_EPI_COLS; ++c) {
                         unsigned code = 0u;
 #pragma unroll
                         for (int k = 0; k < NTHR; ++k) code += (ts[k] < y[c]) ? 1u : 0u;
-                        const int pos = c * BITS;
-                        wv[pos >> 6] |= static_cast<unsigned long long>(code) << (pos & 63);
-                        if ((pos & 63) + BITS > 64) wv[(pos >> 6) + 1] |= static_cast<unsigned long long>(code) >> (64 - (pos & 63));
+                        acc64 |= static_cast<unsigned long long>(code) << filled;
+                        filled += BITS;
+                        if (filled >= 32) {
+                            wv[wi++] = static_cast<uint32_t>(acc64);
+                            acc64 >>= 32;
+                            filled -= 32;
+                        }
                     }
                 } else {
                     constexpr int CPW = 32 / BITS;   // codes per 32-bit word, filled from the top code down
 #pragma unroll
                     for (int k = 0; k < BITS; ++k) {
-                        uint32_t w2[2];
+                        uint32_t w = 0u;
 #pragma unroll
-                        for (int hw = 0; hw < 2; ++hw) {
-                            uint32_t w = 0u;
+                        for (int e = CPW - 1; e >= 0; --e) {
+                            const float v = y[k * CPW + e];
+                            uint32_t code = 0u;
 #pragma unroll
-                            for (int e = CPW - 1; e >= 0; --e) {
-                                const float v = y[(2 * k + hw) * CPW + e];
-                                uint32_t code = 0u;
-#pragma unroll
-                                for (int tt = 0; tt < NTHR; ++tt) code += (ts[tt] < v) ? 1u : 0u;
-                                w = w * (1u << BITS) + code;
-                            }
-                            w2[hw] = w;
+                            for (int tt = 0; tt < NTHR; ++tt) code += (ts[tt] < v) ? 1u : 0u;
+                            w = w * (1u << BITS) + code;
                         }
-                        wv[k] = static_cast<unsigned long long>(w2[0]) | (static_cast<unsigned long long>(w2[1]) << 32);
+                        wv[k] = w;
                     }
                 }
                 const int tok = t * 128 + row;
                 if (tok < n) {
-                    unsigned long long *dst = reinterpret_cast<unsigned long long *>(
-                        out.codes + (static_cast<size_t>(b) * n + tok) * ROW_BYTES + h * 8 * BITS);
+                    uint8_t *dst = out.codes + (static_cast<size_t>(b) * n + tok) * ROW_BYTES + part * 4 * BITS;
+                    if (BITS == 1) *reinterpret_cast<uint32_t *>(dst) = wv[0];
+                    else if (BITS == 2) *reinterpret_cast<uint2 *>(dst) = make_uint2(wv[0], wv[1 % BITS]);
+                    else if (BITS == 4) *reinterpret_cast<uint4 *>(dst) = make_uint4(wv[0], wv[1 % BITS], wv[2 % BITS], wv[3 % BITS]);
+                    else {
 #pragma unroll
-                    for (int k = 0; k < BITS; ++k) dst[k] = wv[k];
-                    if (h == 0) out.norms[static_cast<size_t>(b) * n + tok] = __half_as_ushort(__float2half_rn(rho * (1.0f / Q2_SCALE)));
+                        for (int k = 0; k < BITS; ++k) reinterpret_cast<uint32_t *>(dst)[k] = wv[k];
+                    }
+                    if (part == 0) out.norms[static_cast<size_t>(b) * n + tok] = __half_as_ushort(__float2half_rn(rho * (1.0f / Q2_SCALE)));
                 }
             }
         }
