@@ -99,13 +99,12 @@ static_assert(2 * KPILOT + 9 < EV_EXPL && EV_TOP <= EV_EXPL + 2, "ranks up to 9 
 // With `mark_list` set (first pass over tensor-core Gram matrices), a block whose smallest
 // eigenvalue is not at least REDO_RATIO of the largest (this includes non-finite spectra) is queued
 // in mark_list[atomicAdd(mark_count)] for a second pass with the exact Gram matrix.
-// NT threads: D with FULL (thread t resolves lambda_{t+1}), else 64 (threads 0 .. EV_TOP - 1 resolve
-// lambda_1 .. lambda_EV_TOP, thread EV_TOP the smallest one; lam[EV_TOP .. D-2] is not written).
-template <bool FULL>
+// This is the full-spectrum kernel (D threads, thread t resolves lambda_{t+1}); it serves caches that
+// ask for the `eig` output.
 __device__ __forceinline__ void eigvals_block(const double *__restrict__ diag, const double *__restrict__ off,
                                               double *__restrict__ lam, int blk, int *__restrict__ mark_list,
                                               int *__restrict__ mark_count) {
-    constexpr int NT = FULL ? D : 64, NWARP = NT / 32, PER = D / NT;
+    constexpr int NT = D, NWARP = NT / 32, PER = 1;
     __shared__ __align__(16) double2 sde[D + EV_PAD];
     __shared__ double s_e2[D];
     __shared__ double s_red[3][4];
@@ -202,8 +201,8 @@ __device__ __forceinline__ void eigvals_block(const double *__restrict__ diag, c
     }
     __syncthreads();
     // ascending index of the eigenvalue this thread brackets, and where it goes
-    const bool active = FULL || tid <= EV_TOP;
-    const int slot = FULL ? tid : ((tid < EV_TOP) ? tid : D - 1);   // descending position in lam
+    const bool active = true;
+    const int slot = tid;   // descending position in lam
     const int target = D - 1 - slot;
     int t = -1;                      // largest grid index with count <= target
 #pragma unroll
@@ -277,14 +276,13 @@ __device__ __forceinline__ void eigvals_block(const double *__restrict__ diag, c
     }
 }
 
-template <bool FULL>
-__global__ void __launch_bounds__(FULL ? D : 64) eigvals_kernel(const double *__restrict__ diag, const double *__restrict__ off,
+__global__ void __launch_bounds__(D) eigvals_kernel(const double *__restrict__ diag, const double *__restrict__ off,
                                                                double *__restrict__ lam, const int *__restrict__ list,
                                                                const int *__restrict__ count, int *__restrict__ mark_list,
                                                                int *__restrict__ mark_count) {
     // without a list: block blockIdx.x; with one: the listed blocks, shared out over the grid
     for (int li = blockIdx.x; !list || li < *count; li += gridDim.x) {
-        eigvals_block<FULL>(diag, off, lam, list ? list[li] : li, mark_list, mark_count);
+        eigvals_block(diag, off, lam, list ? list[li] : li, mark_list, mark_count);
         if (!list) break;
         __syncthreads();   // the shared state is reused by the next listed block
     }
@@ -531,17 +529,17 @@ __device__ __forceinline__ void charpoly_sums(const double2 *__restrict__ sde, d
 }
 
 // ------------------------------------------------------------------------------------------
-// Algorithm 2 on the spectrum, then the kept eigenvectors by inverse iteration on the
+// Algorithm 2 on the spectrum, then the kept eigenvectors from the twisted factorisation of the
 // tridiagonal matrix and back-transformation through the stored reflectors.
 // ------------------------------------------------------------------------------------------
 //
 // Every phase here is a chain of dependent latencies (a pivot after a pivot, a reflector after a
 // reflector) that leaves most of the CTA idle, so the kernel is laid out for four CTAs of four warps
-// per SM, whose chains overlap: 12 columns of LU storage (the rank never exceeds the pilot k = 11)
-// and registers for three vectors per warp.
+// per SM, whose chains overlap: 12 columns of factor storage (the rank never exceeds the pilot
+// k = 11) and registers for four vectors per warp.
 constexpr int SP_THREADS = 128, SP_WARPS = SP_THREADS / 32;
-constexpr int LU_LANES = 12;
-static_assert(KPILOT < LU_LANES && KPILOT <= 3 * SP_WARPS, "one LU column and one warp slot per kept vector");
+constexpr int FAC_LANES = 12;
+static_assert(KPILOT < FAC_LANES && KPILOT <= 3 * SP_WARPS, "one factor column and one warp slot per kept vector");
 
 // Back-transformation x = H_0 H_1 ... H_{D-3} y of the kept vectors, normalisation, and the stores of
 // the right singular vectors.  The reflectors (rows of R, 1 KB each) are staged through shared memory
@@ -551,7 +549,7 @@ static_assert(KPILOT < LU_LANES && KPILOT <= 3 * SP_WARPS, "one LU column and on
 // every instruction.  Reflector k is zero up to index k, and whole 16-row chunks of zeros are skipped.
 constexpr int BT_ROWS = 16;                 // reflector rows per stage
 // dynamic shared memory: the vectors, then the two factor arrays or (later) the two reflector stages
-constexpr size_t SPECTRAL_DYN_SMEM = sizeof(double) * (D * LU_LANES + (2 * BT_ROWS * D > 2 * D * LU_LANES ? 2 * BT_ROWS * D : 2 * D * LU_LANES));
+constexpr size_t SPECTRAL_DYN_SMEM = sizeof(double) * (D * FAC_LANES + (2 * BT_ROWS * D > 2 * D * FAC_LANES ? 2 * BT_ROWS * D : 2 * D * FAC_LANES));
 constexpr int BT_BAR_FULL = 2, BT_BAR_EMPTY = 4;   // named barriers: + stage
 
 
@@ -609,8 +607,8 @@ __device__ __forceinline__ void sp_back_transform(const double *__restrict__ R, 
     double y[16];
 #pragma unroll
     for (int m = 0; m < 8; ++m) {
-        y[2 * m] = live ? yv[(16 * m + 2 * sub) * LU_LANES + vi] : 0.0;
-        y[2 * m + 1] = live ? yv[(16 * m + 2 * sub + 1) * LU_LANES + vi] : 0.0;
+        y[2 * m] = live ? yv[(16 * m + 2 * sub) * FAC_LANES + vi] : 0.0;
+        y[2 * m + 1] = live ? yv[(16 * m + 2 * sub + 1) * FAC_LANES + vi] : 0.0;
     }
 #pragma unroll 1
     for (int j = 0; j < NSTAGE; ++j) {
@@ -678,9 +676,9 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
     __shared__ unsigned s_flags;
     extern __shared__ double dyn[];
     double *yv = dyn;                        // D+, then the vectors             [D][12]
-    double *lu_l = dyn + D * LU_LANES;       // e_i / D+_i                       [D][12]
-    double *lu_u = dyn + 2 * D * LU_LANES;   // e_i / D-_{i+1}                   [D][12]
-    double *ring = dyn + D * LU_LANES;       // the back-transformation's reflector stages take the place of lu_l, lu_u
+    double *lu_l = dyn + D * FAC_LANES;       // e_i / D+_i                       [D][12]
+    double *lu_u = dyn + 2 * D * FAC_LANES;   // e_i / D-_{i+1}                   [D][12]
+    double *ring = dyn + D * FAC_LANES;       // the back-transformation's reflector stages take the place of lu_l, lu_u
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = blockIdx.x;
@@ -847,11 +845,11 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
                 if (!(fabs(dp) >= floor_piv)) dp = (dp < 0.0) ? -floor_piv : floor_piv;
                 const double e = ee[i];
                 const double lp = e * sp_rcp(dp);
-                yv[i * LU_LANES + c] = dp;
-                lu_l[i * LU_LANES + c] = lp;
+                yv[i * FAC_LANES + c] = dp;
+                lu_l[i * FAC_LANES + c] = lp;
                 dp = fma(-lp, e, dd[i + 1] - mu);
             }
-            yv[(D - 1) * LU_LANES + c] = dp;
+            yv[(D - 1) * FAC_LANES + c] = dp;
             // backward pivots, and the twist index on the way
             double dm = dd[D - 1] - mu;
             double gbest = fabs(dp);   // gamma_{D-1} = D+_{D-1} (D-_{D-1} is d - mu itself)
@@ -861,10 +859,10 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
                 if (!(fabs(dm) >= floor_piv)) dm = (dm < 0.0) ? -floor_piv : floor_piv;
                 const double e = ee[i];
                 const double um = e * sp_rcp(dm);
-                lu_u[i * LU_LANES + c] = um;
+                lu_u[i * FAC_LANES + c] = um;
                 const double t = dd[i] - mu;
                 dm = fma(-um, e, t);
-                const double gam = fabs(yv[i * LU_LANES + c] + dm - t);
+                const double gam = fabs(yv[i * FAC_LANES + c] + dm - t);
                 if (gam < gbest) {
                     gbest = gam;
                     rbest = i;
@@ -872,17 +870,17 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
             }
             // the vector, left unnormalised (the back-transformation normalises at the end)
             double ss = 1.0;
-            yv[rbest * LU_LANES + c] = 1.0;
+            yv[rbest * FAC_LANES + c] = 1.0;
             double z = 1.0;
             for (int i = rbest - 1; i >= 0; --i) {
-                z = -lu_l[i * LU_LANES + c] * z;
-                yv[i * LU_LANES + c] = z;
+                z = -lu_l[i * FAC_LANES + c] * z;
+                yv[i * FAC_LANES + c] = z;
                 ss = fma(z, z, ss);
             }
             z = 1.0;
             for (int i = rbest; i < D - 1; ++i) {
-                z = -lu_u[i * LU_LANES + c] * z;
-                yv[(i + 1) * LU_LANES + c] = z;
+                z = -lu_u[i * FAC_LANES + c] * z;
+                yv[(i + 1) * FAC_LANES + c] = z;
                 ss = fma(z, z, ss);
             }
             if (!(ss > 0.0 && ss < 1e300)) atomicOr(&s_flags, EOSQ_BLOCK_NOT_CONVERGED);
@@ -924,7 +922,7 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
 
 void launch_eigvals(int64_t nb, const Workspace &ws, const int *list, const int *count, int *mark_list, bool full, cudaStream_t s) {
     if (full) {
-        eigvals_kernel<true><<<list_grid(nb, list), D, 0, s>>>(ws.diag, ws.off, ws.lam, list, count, mark_list, ws.redo_count);
+        eigvals_kernel<<<list_grid(nb, list), D, 0, s>>>(ws.diag, ws.off, ws.lam, list, count, mark_list, ws.redo_count);
     } else {
         const int64_t work = list ? std::min<int64_t>(nb, LIST_GRID) : nb;
         const unsigned grid = static_cast<unsigned>(std::max<int64_t>(1, (work + EVT_WARPS - 1) / EVT_WARPS));

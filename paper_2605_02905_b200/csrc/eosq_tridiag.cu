@@ -77,6 +77,24 @@ __device__ __forceinline__ void tt_sync(int team) {
     else if (team == 2) asm volatile("bar.sync 3, %0;" ::"n"(TEAM_THREADS) : "memory");
     else asm volatile("bar.sync 4, %0;" ::"n"(TEAM_THREADS) : "memory");
 }
+// The sweep token of a CTA with two teams.  Two reductions that share an SM slow each other down
+// most when both sweep at once (the sweep is the one phase that fills the double-precision pipe) and
+// left alone they fall into exactly that rhythm.  So the teams take turns: a team sweeps only while
+// it holds the token and passes it on when its sweep is done; the rest of its step (reductions,
+// barriers, the next reflector) then runs under the other team's sweep.  Barrier 5 carries the token
+// to team 0 and barrier 6 to team 1: the receiver syncs, the giver only arrives.  Both teams take
+// the token the same number of times (a team without work passes it on at once), team 1 gives it
+// away once before its first step, and team 0 takes it once more at the very end.
+template <int TEAM_THREADS>
+__device__ __forceinline__ void tt_token_take(int team) {
+    if (team == 0) asm volatile("bar.sync 5, %0;" ::"n"(2 * TEAM_THREADS) : "memory");
+    else asm volatile("bar.sync 6, %0;" ::"n"(2 * TEAM_THREADS) : "memory");
+}
+template <int TEAM_THREADS>
+__device__ __forceinline__ void tt_token_give(int team) {
+    if (team == 0) asm volatile("bar.arrive 6, %0;" ::"n"(2 * TEAM_THREADS) : "memory");
+    else asm volatile("bar.arrive 5, %0;" ::"n"(2 * TEAM_THREADS) : "memory");
+}
 // 1 / sqrt(x) and 1 / x to a few ulp: the hardware's estimates (about 2^-22) and two Newton steps.
 // Both sit on the chain that every step waits for; x is a sum of squares well inside the normal range
 // (a subnormal or huge x only costs accuracy on a matrix whose scale is already hopeless).
@@ -193,7 +211,7 @@ __device__ __forceinline__ void tt_publish(uint32_t tb, int r, int nxt, int lane
 // first barrier, together with beta_k and gamma_k), p_k, and then, by the warp that holds row k + 1,
 // 2K_k and reflector k + 1.  `trow0` is row 0 of the matrix in global memory; t is the thread's index
 // within its team.
-template <int G, int K0, int TEAMS>
+template <int G, int K0, int TEAMS, bool TOKEN>
 __device__ __forceinline__ void tt_step(uint32_t tb, int k, int kend, int t, int team, TtShared<G> &sh, double *__restrict__ trow0) {
     constexpr int TEAM_THREADS = G * G, NW = TEAM_THREADS / 32;
     const int lane = t & 31, warp = t >> 5, tr = t / G, tc = t & (G - 1);
@@ -227,6 +245,7 @@ __device__ __forceinline__ void tt_step(uint32_t tb, int k, int kend, int t, int
         }
     }
     // The sweep: every live element is brought up to date, written back and used for A u.
+    if (TOKEN) tt_token_take<TEAM_THREADS>(team);
     double acc[8];
     const double *ur = &sh.xu[prv][tr * TT_PSTRIDE], *pr = &sh.pp[prv][tr * TT_PSTRIDE];
 #pragma unroll
@@ -256,6 +275,7 @@ __device__ __forceinline__ void tt_step(uint32_t tb, int k, int kend, int t, int
         tt_st16(tb + 16u * a, raw);
         acc[a] = s0 + s1;
     }
+    if (TOKEN) tt_token_give<TEAM_THREADS>(team);
     // u . A u (parts), then the sums of the partial rows over the G column residues: each stage
     // keeps half of the rows
     double tloc = 0.0;
@@ -323,9 +343,9 @@ __device__ __forceinline__ void tt_step(uint32_t tb, int k, int kend, int t, int
     }
 }
 
-template <int G, int K0, int LO, int HI, int TEAMS>
+template <int G, int K0, int LO, int HI, int TEAMS, bool TOKEN>
 __device__ __forceinline__ void tt_step_if(uint32_t tb, int k, int kend, int t, int team, TtShared<G> &sh, double *__restrict__ trow0) {
-    if constexpr (K0 >= LO && K0 <= HI) tt_step<G, K0, TEAMS>(tb, k, kend, t, team, sh, trow0);
+    if constexpr (K0 >= LO && K0 <= HI) tt_step<G, K0, TEAMS, TOKEN>(tb, k, kend, t, team, sh, trow0);
 }
 
 // Steps [0, KE) of the reduction of the order-8G matrix whose element (i, j) sits at
@@ -333,7 +353,7 @@ __device__ __forceinline__ void tt_step_if(uint32_t tb, int k, int kend, int t, 
 // k goes to row ORIGIN + k (full width, zero up to column ORIGIN + k); diag / off / tau receive
 // d_k, the new off-diagonal entry and gamma_k.  When steps remain the trailing matrix is written
 // back to its own place.  A CTA holds TEAMS teams, each working through its own matrices.
-template <int G, int ORIGIN, int KE, int TEAMS, int MINB>
+template <int G, int ORIGIN, int KE, int TEAMS, int MINB, bool TOKEN>
 __global__ void __launch_bounds__(G *G *TEAMS, MINB) tridiag_tm_kernel(double *__restrict__ gram, double *__restrict__ diag,
                                                                         double *__restrict__ off, double *__restrict__ tau, int nb,
                                                                         const int *__restrict__ list, const int *__restrict__ count) {
@@ -344,6 +364,7 @@ __global__ void __launch_bounds__(G *G *TEAMS, MINB) tridiag_tm_kernel(double *_
     static_assert(LAST || KE % G == 0, "ranges end on tile-slot boundaries");
     static_assert(COLS >= 32 && (COLS & (COLS - 1)) == 0 && COLS <= 512, "tensor-memory allocations are powers of two");
     static_assert(TEAM_THREADS % 32 == 0, "teams are whole warps");
+    static_assert(!TOKEN || TEAMS == 2, "the sweep token goes back and forth between two teams");
     __shared__ __align__(16) TtShared<G> shs[TEAMS];
     __shared__ uint32_t tmem_base_s;
     const int tid = threadIdx.x, cwarp = tid >> 5;
@@ -359,6 +380,7 @@ __global__ void __launch_bounds__(G *G *TEAMS, MINB) tridiag_tm_kernel(double *_
     tc_fence_after_sync();
     const uint32_t tb = tmem_base_s + (static_cast<uint32_t>(32 * (cwarp & 3)) << 16) + 128u * static_cast<uint32_t>(cwarp >> 2);
     const int total = list ? *count : nb;
+    if (TOKEN && team == 1) tt_token_give<TEAM_THREADS>(1);
     for (int li = blockIdx.x * TEAMS + team; li < total; li += gridDim.x * TEAMS) {
         const int blk = list ? list[li] : li;
         double *Gm = gram + static_cast<size_t>(blk) * D * D;
@@ -391,14 +413,14 @@ __global__ void __launch_bounds__(G *G *TEAMS, MINB) tridiag_tm_kernel(double *_
 #pragma unroll 1
         for (int k = 0; k < KE; ++k) {
             switch ((k + 1) / G) {
-                case 0: tt_step_if<G, 0, 0, HI, TEAMS>(tb, k, KE, t, team, sh, T); break;
-                case 1: tt_step_if<G, 1, 0, HI, TEAMS>(tb, k, KE, t, team, sh, T); break;
-                case 2: tt_step_if<G, 2, 0, HI, TEAMS>(tb, k, KE, t, team, sh, T); break;
-                case 3: tt_step_if<G, 3, 0, HI, TEAMS>(tb, k, KE, t, team, sh, T); break;
-                case 4: tt_step_if<G, 4, 0, HI, TEAMS>(tb, k, KE, t, team, sh, T); break;
-                case 5: tt_step_if<G, 5, 0, HI, TEAMS>(tb, k, KE, t, team, sh, T); break;
-                case 6: tt_step_if<G, 6, 0, HI, TEAMS>(tb, k, KE, t, team, sh, T); break;
-                default: tt_step_if<G, 7, 0, HI, TEAMS>(tb, k, KE, t, team, sh, T); break;
+                case 0: tt_step_if<G, 0, 0, HI, TEAMS, TOKEN>(tb, k, KE, t, team, sh, T); break;
+                case 1: tt_step_if<G, 1, 0, HI, TEAMS, TOKEN>(tb, k, KE, t, team, sh, T); break;
+                case 2: tt_step_if<G, 2, 0, HI, TEAMS, TOKEN>(tb, k, KE, t, team, sh, T); break;
+                case 3: tt_step_if<G, 3, 0, HI, TEAMS, TOKEN>(tb, k, KE, t, team, sh, T); break;
+                case 4: tt_step_if<G, 4, 0, HI, TEAMS, TOKEN>(tb, k, KE, t, team, sh, T); break;
+                case 5: tt_step_if<G, 5, 0, HI, TEAMS, TOKEN>(tb, k, KE, t, team, sh, T); break;
+                case 6: tt_step_if<G, 6, 0, HI, TEAMS, TOKEN>(tb, k, KE, t, team, sh, T); break;
+                default: tt_step_if<G, 7, 0, HI, TEAMS, TOKEN>(tb, k, KE, t, team, sh, T); break;
             }
         }
         // The update of the last step is still pending: apply it to what is left of the matrix
@@ -452,6 +474,21 @@ __global__ void __launch_bounds__(G *G *TEAMS, MINB) tridiag_tm_kernel(double *_
         }
         tt_sync<TEAMS, TEAM_THREADS>(team);   // the shared state is reused by the team's next block
     }
+    if (TOKEN) {
+        // Team 0 is never behind team 1 in matrices and at most one ahead: then team 1 passes the
+        // token through once for every step of that matrix.  The last token goes back to team 0.
+        if (team == 1) {
+            const int first0 = blockIdx.x * TEAMS, stride = gridDim.x * TEAMS;
+            const int n0 = first0 < total ? (total - first0 + stride - 1) / stride : 0;
+            const int n1 = first0 + 1 < total ? (total - first0 - 1 + stride - 1) / stride : 0;
+            for (int i = 0; i < (n0 - n1) * KE; ++i) {
+                tt_token_take<TEAM_THREADS>(1);
+                tt_token_give<TEAM_THREADS>(1);
+            }
+        } else {
+            tt_token_take<TEAM_THREADS>(0);
+        }
+    }
     tc_fence_before_sync();
     __syncthreads();
     if (cwarp == 0) {
@@ -470,11 +507,11 @@ void launch_tridiag(int part, int64_t nb, const Workspace &ws, const int *list, 
     const int n = static_cast<int>(nb);
     const int64_t work = list ? std::min<int64_t>(nb, LIST_GRID) : nb;
     if (part == 0) {
-        const int grid = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(work, 2 * static_cast<int64_t>(sm_count))));
-        tridiag_tm_kernel<16, 0, 64, 1, 2><<<grid, 256, 0, s>>>(g0, d0, o0, t0, n, list, count);
+        const int grid = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>((work + 1) / 2, static_cast<int64_t>(sm_count))));
+        tridiag_tm_kernel<16, 0, 64, 2, 1, true><<<grid, 512, 0, s>>>(g0, d0, o0, t0, n, list, count);
     } else {
         const int grid = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>((work + 1) / 2, 4 * static_cast<int64_t>(sm_count))));
-        tridiag_tm_kernel<8, 64, 62, 2, 4><<<grid, 128, 0, s>>>(g0, d0, o0, t0, n, list, count);
+        tridiag_tm_kernel<8, 64, 62, 2, 4, false><<<grid, 128, 0, s>>>(g0, d0, o0, t0, n, list, count);
     }
 }
 
