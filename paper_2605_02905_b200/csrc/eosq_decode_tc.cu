@@ -50,6 +50,22 @@ __device__ __forceinline__ uint32_t dt_offset(int row, int jc) {
 __device__ __forceinline__ void dt_bar_sync(int half) {
     asm volatile("bar.sync %0, %1;" ::"r"(1 + half), "r"(DT_HALF) : "memory");
 }
+// The same barrier, telling every thread of the half whether any of them brings `failed`.  A bounded
+// wait ends per thread, so one thread may give up where its neighbour just succeeds: the outcome is
+// made common here, at the next barrier of the half, and the half leaves its loop as a whole (a
+// thread that left alone would let this barrier wait for ever).
+__device__ __forceinline__ bool dt_bar_any(int half, bool failed) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 p, %1, 0;\n\t"
+        "bar.red.or.pred q, %2, %3, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(r)
+        : "r"(failed ? 1u : 0u), "r"(1 + half), "r"(DT_HALF)
+        : "memory");
+    return r != 0;
+}
 
 struct DecodeArgs {
     eosq_cache_t cache;
@@ -170,10 +186,9 @@ __global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeAr
         for (int tile = 0; tile < tiles; ++tile) {
             const bool valid = tile * 128 + r < n;
             // the tile's raw data (asked for one tile ago); rows past the end of the block were not copied
-            if (!mbar_wait(&raw_full[half], raw_phase, &abort_flag)) {
-                alive = false;
-                break;
-            }
+            // (a thread whose wait gave up works on with whatever the raw area holds, up to the barrier
+            // below the operand stores, where the half learns of it)
+            const bool raw_ok = mbar_wait(&raw_full[half], raw_phase, &abort_flag);
             raw_phase ^= 1u;
             uint32_t cw[2 * BITS];
 #pragma unroll
@@ -214,7 +229,11 @@ __global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeAr
             }
             const float f = __half2float(__ushort_as_half(static_cast<unsigned short>(rho_raw))) * a.inv_scale;
             fence_proxy_async_smem();   // the operands were written by ordinary stores and are read by the tensor core
-            dt_bar_sync(half);
+            if (dt_bar_any(half, !raw_ok)) {
+                alive = false;
+                raw_phase ^= 1u;   // the phase that did not complete is the one the final drain waits for
+                break;
+            }
             if (ht == 0) {
                 tc_fence_after_sync();
                 constexpr uint32_t idesc = umma_idesc_f16(128, D, false, false);
@@ -233,10 +252,9 @@ __global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeAr
                 if (tile + 1 < tiles) issue(blk, tile + 1, rank);
                 else if (blk + bstep < a.nb) issue(blk + bstep, 0, rank_next);
             }
-            if (!mbar_wait(&mma_done[half], phase, &abort_flag)) {
-                alive = false;
-                break;
-            }
+            // (likewise: a thread that gave up reads accumulators that may not be final, and the barrier
+            // behind the epilogue ends the loop for the whole half before anything of the tile is stored)
+            const bool mma_ok = mbar_wait(&mma_done[half], phase, &abort_flag);
             phase ^= 1u;
             tc_fence_after_sync();
             const int tok = tile * 128 + r;
@@ -277,7 +295,10 @@ __global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeAr
             if (sizeof(Tout) == 2) {
                 fence_proxy_async_smem();   // the staged tile was written by ordinary stores and is read by the copy engine
                 tc_fence_before_sync();
-                dt_bar_sync(half);
+                if (dt_bar_any(half, !mma_ok)) {
+                    alive = false;
+                    break;
+                }
                 if (ht == 0) {
                     tma_store_3d(&omap, hbase + DT_H_A, 0, tile * 128, static_cast<int>(blk));
                     tma_store_3d(&omap, hbase + DT_H_A + DT_BOX, 64, tile * 128, static_cast<int>(blk));
@@ -286,7 +307,10 @@ __global__ void __launch_bounds__(DT_THREADS, 1) decode_tc_kernel(const DecodeAr
                 store_pending = true;   // waited for before the tile is overwritten
             } else {
                 tc_fence_before_sync();
-                dt_bar_sync(half);   // operands and accumulators are free for the next tile
+                if (dt_bar_any(half, !mma_ok)) {   // operands and accumulators are free for the next tile
+                    alive = false;
+                    break;
+                }
             }
         }
     }

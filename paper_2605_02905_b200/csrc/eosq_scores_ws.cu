@@ -81,6 +81,21 @@ __device__ __forceinline__ void ws_split_store(uint8_t *plane, int g, int k, flo
     *reinterpret_cast<__half *>(plane + ws_b_offset(WS_NQ + g, k)) = lo;
 }
 
+// Barrier of the 64 threads of the operand builder that also tells each of them whether any brings
+// `failed` (the outcome of a bounded wait, which ends per thread).
+__device__ __forceinline__ bool ws_builder_any(bool failed) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 p, %1, 0;\n\t"
+        "bar.red.or.pred q, 2, 64, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(r)
+        : "r"(failed ? 1u : 0u)
+        : "memory");
+    return r != 0;
+}
+
 struct WsBarriers {
     uint64_t st_full[WS_STAGES], st_empty[WS_STAGES];
     uint64_t a_full[WS_BUFS], d_full[WS_BUFS], d_empty[WS_BUFS];
@@ -283,8 +298,10 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
         auto build_w = [&](int hd, int hx) -> bool {
             const int hb = hx & 1;
             float *qs = qs_all + hb * WS_NQ * D;
-            if (!mbar_wait(&bars.b1_empty[hb], ((hx >> 1) & 1u) ^ 1u, &abort_flag)) return false;
-            if (bt == 0) {
+            // (a bounded wait ends per thread: its outcome is made common at the group's next barrier, so
+            // that the 64 threads leave together and never one by one)
+            const bool ok = mbar_wait(&bars.b1_empty[hb], ((hx >> 1) & 1u) ^ 1u, &abort_flag);
+            if (bt == 0 && ok) {
                 mbar_arrive_expect_tx(&bars.b1_full[hb], 4096);
                 ws_bulk_load(base + L::OFF_B1 + hb * 4096, a.wimg + static_cast<size_t>(hd) * 4096, 4096, &bars.b1_full[hb]);
             }
@@ -292,8 +309,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
                 const int g = e / D;
                 qs[e] = (g < gcount) ? __half2float(a.q[(static_cast<long long>(hd) * a.G + a.g0 + g) * D + (e % D)]) : 0.0f;
             }
-            asm volatile("bar.sync 2, 64;" ::: "memory");
-            return true;
+            return !ws_builder_any(!ok);
         };
         int head = (it0 < it1) ? it0 / a.bph : 0, jb = it0 - head * a.bph, hidx = -1, prev_head = -1;
         bool first_of_head = false;
@@ -306,7 +322,6 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
                 if (hidx == 0 && !build_w(head, 0)) break;   // later heads were built one head ahead (below)
             }
             const float *qs = qs_all + (hidx & 1) * WS_NQ * D;
-            const long long gb = static_cast<long long>(head) * a.head_stride + jb;
             const int vb = bi & 1;
             const int rank = rank_next;
             {   // the next block's rank is asked for now: a load on the critical path of every block costs over 1 000 cycles
@@ -317,9 +332,8 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
                 }
                 if (item + 1 < it1) rank_next = min(__ldg(a.cache.rank + static_cast<long long>(nh) * a.head_stride + nj), WS_PMAX);
             }
-            if (!mbar_wait(&bars.blk_full[vb], (bi >> 1) & 1u, &abort_flag) ||
-                !mbar_wait(&bars.b2_empty[vb], ((bi >> 1) & 1u) ^ 1u, &abort_flag))
-                break;
+            const bool ok = mbar_wait(&bars.blk_full[vb], (bi >> 1) & 1u, &abort_flag) &&
+                            mbar_wait(&bars.b2_empty[vb], ((bi >> 1) & 1u) ^ 1u, &abort_flag);
             const __half *vs = reinterpret_cast<const __half *>(base + L::OFF_V + vb * 4096);
             uint8_t *b2 = base + L::OFF_B2 + vb * 2048;
             // Aq[g][i] = q_g . zeta_i for g < gcount, i < rank, zero elsewhere.  Four lanes share a dot product
@@ -361,7 +375,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) scores_ws_kernel(const WsArgs a
                 if (act && part == 0) ws_split_store(b2, g, i, dot * WS_QSCALE);
             }
             fence_proxy_async_smem();
-            asm volatile("bar.sync 2, 64;" ::: "memory");
+            if (ws_builder_any(!ok)) break;   // a thread whose wait gave up has built from stale vectors: nothing is handed on
             if (bt == 0) {
                 mbar_arrive(&bars.b2_full[vb]);
                 mbar_arrive(&bars.blk_empty[vb]);
