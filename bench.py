@@ -54,13 +54,27 @@ def measured_peaks():
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
 
 
-def recorded_traffic():
-    """DRAM bytes per block of each kernel from the committed ncu capture (profiles/traffic.json), or {}."""
+def recorded_traffic(n: int, d: int, bits: int):
+    """DRAM bytes per block of each kernel from the committed ncu capture (profiles/traffic.json).  The
+    record names the kernel sources it was taken on (a hash over csrc/) and the block shape; when either
+    differs from what runs now the counters no longer describe it and {} is returned (traffic: null)."""
+    import glob
+    import hashlib
     path = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(path):
-        with open(path) as f:
-            return json.load(f)
-    return {}
+    if not os.path.exists(path):
+        return {}
+    with open(path) as f:
+        rec = json.load(f)
+    h = hashlib.sha256()
+    for src in sorted(glob.glob(os.path.join(ROOT, "paper_2605_02905_b200", "csrc", "*"))):
+        h.update(os.path.basename(src).encode())
+        with open(src, "rb") as f:
+            h.update(f.read())
+    if h.hexdigest() != rec.get("sources_sha256"):
+        return {"note": "the kernels have changed since the recorded ncu capture"}
+    if (n, d, bits) != (1024, 128, 2):
+        return {"note": "the recorded ncu capture is of n = 1024, d = 128, b = 2"}
+    return rec
 
 
 class ClockSampler:
@@ -417,7 +431,7 @@ def run_library(args):
     # Gram + rotation flops at the tensor peak.  The double-precision spectral stages are credited nothing.
     roof_ms, roof_bound = encode_roofline_ms(peaks, in_bytes, B * out_bytes_per_block, B, n, d)
     algo_bytes = in_bytes + B * out_bytes_per_block
-    traffic_tab = recorded_traffic()
+    traffic_tab = recorded_traffic(n, d, args.bits)
     roofline = {"kernel": "eosq_encode (all stages of one pass)", "bound": roof_bound,
                 "achieved": (algo_bytes / (enc_ms * 1e-3) / 1e9) if roof_bound == "hbm" else (B * 4.0 * n * d * d / (enc_ms * 1e-3) / 1e12),
                 "peak": peaks["hbm_gbs"] if roof_bound == "hbm" else peaks["bf16_tflops_sustained"],
@@ -434,7 +448,7 @@ def run_library(args):
         # Householder tridiagonalisation: 4/3 m^3 flops for order m; two kernels take d -> d/2 -> 0
         "tridiag_a": ("alu", (4.0 / 3.0) * (d ** 3 - (d // 2) ** 3) / 1e12, FP64_NOMINAL_TFLOPS, "TFLOP/s", "nominal (SMs x lanes x clock)"),
         "tridiag_b": ("alu", (4.0 / 3.0) * (d // 2) ** 3 / 1e12, FP64_NOMINAL_TFLOPS, "TFLOP/s", "nominal (SMs x lanes x clock)"),
-        "eigvals": ("alu", 16 * (3 * 11 + 2) * d * 6.0 / 1e12, FP64_NOMINAL_TFLOPS, "TFLOP/s", "nominal (SMs x lanes x clock)"),
+        "eigvals": ("alu", 32 * 14 * d * 6.0 / 1e12, FP64_NOMINAL_TFLOPS, "TFLOP/s", "nominal (SMs x lanes x clock)"),
         "spectral": ("alu", (4.0 * d * d * max(mean_rank, 1.0)) / 1e12, FP64_NOMINAL_TFLOPS, "TFLOP/s", "nominal (SMs x lanes x clock)"),
         "quant": ("hbm", (n * d * 2 + out_bytes_per_block) / 1e9, peaks["hbm_gbs"], "GB/s", peaks["source"]),
     }

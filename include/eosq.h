@@ -208,9 +208,20 @@ int eosq_encode_host(eosq_ctx *ctx, const void *host_blocks, int in_dtype, int64
                      size_t arena_bytes, void *cuda_stream);
 
 /* Synchronises the stream and returns EOSQ_WARN_BLOCK_STATUS if any of the num_blocks status
- * words (dev) is non-zero, EOSQ_OK otherwise; *flagged (host, may be null) gets the count. */
+ * words (dev) is non-zero, EOSQ_OK otherwise; *flagged (host, may be null) gets the count.
+ * If a kernel launched through the context has given up a bounded device-side wait since the last
+ * call (its outputs are then incomplete), returns EOSQ_ERR_CUDA instead, with the kernels' bits in
+ * eosq_last_cuda_error() (1 Gram, 2 quantise, 8 scores, 16 decode, 32 self-test), and clears that
+ * record: it is reported once and the context stays usable. */
 int eosq_check_status(eosq_ctx *ctx, const int32_t *status, int64_t num_blocks, int64_t *flagged,
                       void *cuda_stream);
+
+/* Launches a one-CTA kernel that waits on a barrier nothing arrives at, for at most `polls`
+ * (1..4096) polls of about 2 us, gives up and records that like any pipeline kernel of the library
+ * would: the next eosq_check_status returns EOSQ_ERR_CUDA (bit 32).  No output, no effect on cache
+ * data; it exists so that the time-out path can be exercised without a kernel that hangs or faults.
+ * EOSQ_ERR_INVALID_ARG for polls outside the range. */
+int eosq_selftest_wait_timeout(eosq_ctx *ctx, uint32_t polls, void *cuda_stream);
 
 /* Number of kernels the library has launched through this context so far (for bookkeeping). */
 int64_t eosq_launch_count(const eosq_ctx *ctx);

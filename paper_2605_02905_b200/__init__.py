@@ -27,7 +27,7 @@ EXPORTS = [
     "eosq_workspace_bytes", "eosq_create", "eosq_destroy", "eosq_last_cuda_error", "eosq_encode",
     "eosq_decode", "eosq_scores", "eosq_encode_host_arena_bytes", "eosq_encode_host",
     "eosq_check_status", "eosq_launch_count", "eosq_profile_enable", "eosq_profile_select", "eosq_profile_read",
-    "eosq_encode_static", "eosq_encode_static_max_blocks",
+    "eosq_encode_static", "eosq_encode_static_max_blocks", "eosq_selftest_wait_timeout",
 ]
 STAGES = ["gram", "tridiag_a", "tridiag_b", "eigvals", "spectral", "quant", "decode", "scores", "redo", "other"]
 
@@ -90,6 +90,7 @@ def lib():
                                   ctypes.c_void_p, ctypes.c_void_p]
         L.eosq_encode_host.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
                                        ctypes.c_int, ctypes.c_uint64, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+        L.eosq_selftest_wait_timeout.argtypes = [ctypes.c_void_p, ctypes.c_uint32, ctypes.c_void_p]
         L.eosq_profile_enable.argtypes = [ctypes.c_void_p, ctypes.c_int]
         L.eosq_profile_select.argtypes = [ctypes.c_void_p, ctypes.c_uint32]
         L.eosq_profile_read.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
@@ -163,6 +164,10 @@ class Context:
             self.close()
         except Exception:
             pass
+
+    def selftest_wait_timeout(self, polls: int = 64, stream=None):
+        """Launches the kernel whose bounded wait runs out; the next check_status reports it."""
+        _check(lib().eosq_selftest_wait_timeout(self._h, int(polls), _stream_ptr(stream)), "eosq_selftest_wait_timeout", self)
 
     @property
     def launch_count(self) -> int:

@@ -517,10 +517,23 @@ extern "C" int eosq_check_status(eosq_ctx *ctx, const int32_t *status, int64_t n
     if (record_cuda(ctx, cudaStreamSynchronize(s), "cudaStreamSynchronize")) return EOSQ_ERR_CUDA;
     if (dev_err != 0) {
         ctx->last_error = "a bounded device-side wait gave up (kernel bits " + std::to_string(dev_err) + "); results are incomplete";
+        // reported once: the word is cleared so that the context can be used again
+        if (record_cuda(ctx, cudaMemsetAsync(ctx->dev_err, 0, sizeof(int), s), "error word reset") ||
+            record_cuda(ctx, cudaStreamSynchronize(s), "cudaStreamSynchronize"))
+            return EOSQ_ERR_CUDA;
+        ctx->last_error = "a bounded device-side wait gave up (kernel bits " + std::to_string(dev_err) + "); results are incomplete";
         return EOSQ_ERR_CUDA;
     }
     int64_t cnt = 0;
     for (int32_t v : h) cnt += (v != 0);
     if (flagged) *flagged = cnt;
     return cnt ? EOSQ_WARN_BLOCK_STATUS : EOSQ_OK;
+}
+
+extern "C" int eosq_selftest_wait_timeout(eosq_ctx *ctx, uint32_t polls, void *cuda_stream) {
+    if (!ctx || polls == 0 || polls > 4096 || !on_ctx_device(ctx)) return EOSQ_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    launch_wait_timeout(ctx->dev_err, polls, s);
+    ctx->launches += 1;
+    return record_cuda(ctx, cudaGetLastError(), "eosq_selftest_wait_timeout launch") ? EOSQ_ERR_CUDA : EOSQ_OK;
 }

@@ -184,4 +184,6 @@ __device__ __forceinline__ float load_as_float<float>(const float *p) { return *
 template <>
 __device__ __forceinline__ float load_as_float<__half>(const __half *p) { return __half2float(*p); }
 
+void launch_wait_timeout(int *err, uint32_t polls, cudaStream_t s);
+
 }  // namespace eosq

@@ -53,18 +53,21 @@ __device__ __forceinline__ bool mbar_test_wait(uint64_t *bar, uint32_t parity) {
 
 constexpr uint32_t WAIT_POLLS = 1u << 20;  // each poll suspends for at most ~2 us: a wait gives up after about 2 s
 
-// Waits for the phase with the given parity to complete.  Returns false if it gave up, either
-// because the poll budget ran out (it then raises *abort_flag) or because another thread of the
-// CTA raised *abort_flag.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
+// Waits for the phase with the given parity to complete, for at most `polls` blocking polls.  Returns
+// false if it gave up, either because the poll budget ran out (it then raises *abort_flag) or because
+// another thread of the CTA raised *abort_flag.
+__device__ __forceinline__ bool mbar_wait_limited(uint64_t *bar, uint32_t parity, volatile int *abort_flag, uint32_t polls) {
     if (mbar_test_wait(bar, parity)) return true;   // the common case in a pipeline that runs ahead
-    for (uint32_t it = 0; it < WAIT_POLLS; ++it) {
+    for (uint32_t it = 0; it < polls; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 63u) == 63u && *abort_flag) return false;
         if (it >= 64) __nanosleep(64);   // a long wait backs off; a hand-over between pipeline stages must not oversleep
     }
     *abort_flag = 1;
     return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
+    return mbar_wait_limited(bar, parity, abort_flag, WAIT_POLLS);
 }
 
 // ---- proxies and fences ----------------------------------------------------------------------

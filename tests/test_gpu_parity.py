@@ -429,3 +429,25 @@ def test_unaligned_cache_arrays_are_rejected(ctx):
     rc = L.eosq_scores(ctx._h, ctypes.addressof(st), 1, 2, 2, 256, 128, 2, ctypes.c_uint64(SEED), q.data_ptr(), 4,
                        ctypes.c_float(0.1), s.data_ptr(), stream)
     assert rc == eosq.EOSQ_ERR_INVALID_ARG
+
+
+def test_a_wait_that_runs_out_is_reported_once_and_the_context_stays_usable(ctx):
+    """The time-out path without a hang: a kernel waits (a few hundred microseconds at most) on a barrier
+    nothing arrives at, gives up, and the context reports it as an error of the next status check; after
+    that the same context compresses as before."""
+    w = synth.kv_cache_blocks("timeout", layers=1, kv_heads=2, tokens=512, n=256, rank_hi=4, seed=77)
+    blocks = w.blocks.cuda()
+    before = eosq.eosq_encode(ctx, blocks, 2, SEED)
+    assert eosq.eosq_check_status(ctx, before) == 0
+    L = eosq.lib()
+    assert L.eosq_selftest_wait_timeout(ctx._h, 0, None) == eosq.EOSQ_ERR_INVALID_ARG
+    assert L.eosq_selftest_wait_timeout(ctx._h, 5000, None) == eosq.EOSQ_ERR_INVALID_ARG
+    ctx.selftest_wait_timeout(polls=128)
+    with pytest.raises(eosq.EosqError) as err:
+        eosq.eosq_check_status(ctx, before)
+    assert err.value.code == eosq.EOSQ_ERR_CUDA and "kernel bits 32" in str(err.value)
+    assert eosq.eosq_check_status(ctx, before) == 0          # reported once
+    after = eosq.eosq_encode(ctx, blocks, 2, SEED)
+    assert eosq.eosq_check_status(ctx, after) == 0
+    for name in ("codes", "norms", "rank", "sigma", "phi", "V", "status"):
+        assert torch.equal(getattr(before, name), getattr(after, name)), name

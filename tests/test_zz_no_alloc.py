@@ -10,6 +10,8 @@ run every other test.
 """
 import ctypes
 
+import gc
+
 import pytest
 import torch
 
@@ -61,6 +63,7 @@ def test_static_scratch_encode_matches_workspace_encode_twice():
             # caching allocator nor the driver may have been asked for a byte
             for name in FIELDS + ("P",):
                 getattr(out, name).fill_(0)
+            gc.collect()   # tensors that earlier tests left in reference cycles go now, not during the call
             torch.cuda.synchronize()
             alloc0, reserved0, used0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved(), _device_bytes_in_use()
             eosq.eosq_encode_static(ctx, dev, bits, seed, out)
