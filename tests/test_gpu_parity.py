@@ -299,6 +299,40 @@ def test_full_size_cache_sampled_blocks(ctx, bits, full):
     parity.compare_decode(sub_cache, dec[pick], bits, SEED, tol=1e-3)
 
 
+def test_full_size_ministral_cache_sampled_blocks(ctx):
+    """Config 3 at its full size and in the benchmark's launch configuration: the Ministral-8B-shaped 64k
+    cache (36864 blocks, 9 GiB; two chunks of the library's scratch) is encoded at b = 2 in one call, the
+    logits of G = 16 queries per KV head (4 query heads x batch 4) are taken against compressed keys, and
+    blocks sampled on both sides of the chunk boundary go to the oracle one by one."""
+    w = synth.ministral_64k(device="cuda")
+    B = w.blocks.shape[0]
+    assert B == 36864
+    cache = eosq.Cache.allocate(B, w.n, w.d, 2, diagnostics="staged")
+    eosq.eosq_encode(ctx, w.blocks, 2, SEED, out=cache)
+    torch.cuda.synchronize()
+    assert eosq.eosq_check_status(ctx, cache) == 0
+    ranks = cache.rank
+    assert int(ranks.min()) >= 0 and int(ranks.max()) <= 11
+    assert torch.all(torch.isfinite(cache.norms.float()))
+    planted = w.planted_rank
+    noise_values = [i for i in range(B) if planted[i] == 0 and not bool(w.is_key[i])]
+    assert noise_values and all(int(ranks[i]) == 0 for i in noise_values[:200])
+    pick = sorted({0, 63, 64, 18943, 18944, 18945, 30001, B - 1, noise_values[0]})
+    sub = w.blocks[pick].cpu()
+    sub_cache = eosq.Cache.allocate(len(pick), w.n, w.d, 2, diagnostics="staged")
+    for name in ("codes", "norms", "rank", "sigma", "phi", "P", "V", "status", "lambda_plus", "vr32", "coef"):
+        getattr(sub_cache, name).copy_(getattr(cache, name)[pick])
+    rep, enc = parity.compare_encode(sub, sub_cache, 2, SEED)
+    _report("ministral_64k_sampled_b2", rep)
+    assert rep["e2e_out_band_fraction"] < 1e-4
+    heads, bph, G = 8, 64, 16
+    q = synth.queries(heads, G, seed=9).cuda()
+    s = eosq.eosq_scores(ctx, cache, q, heads, bph, 2 * bph, SEED)
+    torch.cuda.synchronize()
+    assert eosq.eosq_check_status(ctx, cache) == 0
+    parity.compare_scores(cache, q, s, heads, bph, 2 * bph, 2, SEED, 1.0 / math.sqrt(128), pairs=[(0, 0), (3, 40), (7, 63)])
+
+
 def _stratified(planted, is_key, want):
     """Indices of blocks covering the planted ranks in `want` for keys and values (first match each)."""
     pick = []
