@@ -19,6 +19,8 @@ bool eosq::ensure_dynamic_smem(const void *kernel, size_t bytes) {
     for (const auto &e : done)
         if (e.first == kernel && e.second == dev) return true;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes)) != cudaSuccess) return false;
+    // every kernel that comes here sizes its CTAs per SM by shared memory: ask for all of it
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) != cudaSuccess) return false;
     done.emplace_back(kernel, dev);
     return true;
 }

@@ -535,21 +535,26 @@ __device__ __forceinline__ void charpoly_sums(const double2 *__restrict__ sde, d
 //
 // Every phase here is a chain of dependent latencies (a pivot after a pivot, a reflector after a
 // reflector) that leaves most of the CTA idle, so the kernel is laid out for four CTAs of four warps
-// per SM, whose chains overlap: 12 columns of factor storage (the rank never exceeds the pilot
-// k = 11) and registers for four vectors per warp.
+// per SM, whose chains overlap (measured: 3.4 / 2.4 / 1.9 ms at two / three / four CTAs per SM).
+// Shared memory (33 KB: 12 columns of factor storage - the rank never exceeds the pilot k = 11 - in
+// two arrays that the vectors and the reflector stages take over in turn) would allow six, but the
+// 80 or 90 registers per thread that five or six CTAs leave cost more than the extra CTAs bring
+// (2.5 ms against 1.8 ms).
 constexpr int SP_THREADS = 128, SP_WARPS = SP_THREADS / 32;
 constexpr int FAC_LANES = 12;
 static_assert(KPILOT < FAC_LANES && KPILOT <= 3 * SP_WARPS, "one factor column and one warp slot per kept vector");
 
 // Back-transformation x = H_0 H_1 ... H_{D-3} y of the kept vectors, normalisation, and the stores of
 // the right singular vectors.  The reflectors (rows of R, 1 KB each) are staged through shared memory
-// by the CTA's last warp, sixteen rows per stage and two stages, handed over with named barriers.
+// by the CTA's last warp, six rows per stage and two stages, handed over with named barriers.
 // The other three warps apply them: a group of eight lanes owns one vector (sixteen entries per
 // lane: rows 16 m + 2 sub, + 1), so a dot product needs three shuffle stages and four vectors share
 // every instruction.  Reflector k is zero up to index k, and whole 16-row chunks of zeros are skipped.
-constexpr int BT_ROWS = 16;                 // reflector rows per stage
-// dynamic shared memory: the vectors, then the two factor arrays or (later) the two reflector stages
-constexpr size_t SPECTRAL_DYN_SMEM = sizeof(double) * (D * FAC_LANES + (2 * BT_ROWS * D > 2 * D * FAC_LANES ? 2 * BT_ROWS * D : 2 * D * FAC_LANES));
+constexpr int BT_ROWS = 6;                  // reflector rows per stage: two stages fill one factor array
+static_assert((D - 2) % BT_ROWS == 0 && 2 * BT_ROWS * D <= D * FAC_LANES, "the stages take the place of the second factor array");
+// dynamic shared memory: two arrays [D][12].  The first holds e_i / D+_i and then, in place, the vectors;
+// the second D+_i, then e_i / D-_{i+1}, then the two reflector stages.
+constexpr size_t SPECTRAL_DYN_SMEM = sizeof(double) * 2 * D * FAC_LANES;
 constexpr int BT_BAR_FULL = 2, BT_BAR_EMPTY = 4;   // named barriers: + stage
 
 
@@ -675,10 +680,9 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
     __shared__ double s_phi[RMAX], s_sig[RMAX];
     __shared__ unsigned s_flags;
     extern __shared__ double dyn[];
-    double *yv = dyn;                        // D+, then the vectors             [D][12]
-    double *lu_l = dyn + D * FAC_LANES;       // e_i / D+_i                       [D][12]
-    double *lu_u = dyn + 2 * D * FAC_LANES;   // e_i / D-_{i+1}                   [D][12]
-    double *ring = dyn + D * FAC_LANES;       // the back-transformation's reflector stages take the place of lu_l, lu_u
+    double *yv = dyn;                        // e_i / D+_i, then the vectors                       [D][12]
+    double *fb = dyn + D * FAC_LANES;         // D+_i, then e_i / D-_{i+1}                          [D][12]
+    double *ring = dyn + D * FAC_LANES;       // the back-transformation's reflector stages take the place of fb
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = blockIdx.x;
@@ -838,18 +842,17 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
         if (warp == 0 && lane < rank) {
             const int c = lane;
             const double mu = lam[c];
-            // forward pivots; yv keeps D+ until the vector takes its place
+            // forward pivots: the ratios go where the vector will be, D+ where the backward ratios will be
             double dp = dd[0] - mu;
 #pragma unroll 4
             for (int i = 0; i < D - 1; ++i) {
                 if (!(fabs(dp) >= floor_piv)) dp = (dp < 0.0) ? -floor_piv : floor_piv;
                 const double e = ee[i];
                 const double lp = e * sp_rcp(dp);
-                yv[i * FAC_LANES + c] = dp;
-                lu_l[i * FAC_LANES + c] = lp;
+                fb[i * FAC_LANES + c] = dp;
+                yv[i * FAC_LANES + c] = lp;
                 dp = fma(-lp, e, dd[i + 1] - mu);
             }
-            yv[(D - 1) * FAC_LANES + c] = dp;
             // backward pivots, and the twist index on the way
             double dm = dd[D - 1] - mu;
             double gbest = fabs(dp);   // gamma_{D-1} = D+_{D-1} (D-_{D-1} is d - mu itself)
@@ -859,10 +862,11 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
                 if (!(fabs(dm) >= floor_piv)) dm = (dm < 0.0) ? -floor_piv : floor_piv;
                 const double e = ee[i];
                 const double um = e * sp_rcp(dm);
-                lu_u[i * FAC_LANES + c] = um;
+                const double dpi = fb[i * FAC_LANES + c];   // D+_i, read before its place is taken
+                fb[i * FAC_LANES + c] = um;
                 const double t = dd[i] - mu;
                 dm = fma(-um, e, t);
-                const double gam = fabs(yv[i * FAC_LANES + c] + dm - t);
+                const double gam = fabs(dpi + dm - t);
                 if (gam < gbest) {
                     gbest = gam;
                     rbest = i;
@@ -873,13 +877,13 @@ __global__ void __launch_bounds__(SP_THREADS, 4) spectral_kernel(int n, Workspac
             yv[rbest * FAC_LANES + c] = 1.0;
             double z = 1.0;
             for (int i = rbest - 1; i >= 0; --i) {
-                z = -lu_l[i * FAC_LANES + c] * z;
+                z = -yv[i * FAC_LANES + c] * z;   // the ratio's place becomes the entry's
                 yv[i * FAC_LANES + c] = z;
                 ss = fma(z, z, ss);
             }
             z = 1.0;
             for (int i = rbest; i < D - 1; ++i) {
-                z = -lu_u[i * FAC_LANES + c] * z;
+                z = -fb[i * FAC_LANES + c] * z;
                 yv[(i + 1) * FAC_LANES + c] = z;
                 ss = fma(z, z, ss);
             }
