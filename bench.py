@@ -311,7 +311,7 @@ def run_library(args):
         if num_heads > 0:
             eosq.eosq_scores(ctx, cache, q, num_heads, bph, 2 * bph, SEED, out=scores)
 
-    ENC_STAGES = ("gram", "tridiag_a", "tridiag_b", "eigvals", "spectral", "quant", "redo")
+    ENC_STAGES = ("gram", "tridiag_a", "tridiag_b", "tridiag_c", "eigvals", "spectral", "quant", "redo")
     for _ in range(max(args.warmup, 3)):
         step()
     torch.cuda.synchronize()
@@ -445,9 +445,10 @@ def run_library(args):
     # the kernel with the largest share, against the bound that holds for it
     algo = {
         "gram": ("tensor", 2.0 * n * d * d / 1e12, peaks["bf16_tflops_sustained"], "TFLOP/s", peaks["source"]),
-        # Householder tridiagonalisation: 4/3 m^3 flops for order m; two kernels take d -> d/2 -> 0
+        # Householder tridiagonalisation: 4/3 m^3 flops for order m; three kernels take d -> d/2 -> d/4 -> 0
         "tridiag_a": ("alu", (4.0 / 3.0) * (d ** 3 - (d // 2) ** 3) / 1e12, FP64_NOMINAL_TFLOPS, "TFLOP/s", "nominal (SMs x lanes x clock)"),
-        "tridiag_b": ("alu", (4.0 / 3.0) * (d // 2) ** 3 / 1e12, FP64_NOMINAL_TFLOPS, "TFLOP/s", "nominal (SMs x lanes x clock)"),
+        "tridiag_b": ("alu", (4.0 / 3.0) * ((d // 2) ** 3 - (d // 4) ** 3) / 1e12, FP64_NOMINAL_TFLOPS, "TFLOP/s", "nominal (SMs x lanes x clock)"),
+        "tridiag_c": ("alu", (4.0 / 3.0) * (d // 4) ** 3 / 1e12, FP64_NOMINAL_TFLOPS, "TFLOP/s", "nominal (SMs x lanes x clock)"),
         "eigvals": ("alu", 32 * 14 * d * 6.0 / 1e12, FP64_NOMINAL_TFLOPS, "TFLOP/s", "nominal (SMs x lanes x clock)"),
         "spectral": ("alu", (4.0 * d * d * max(mean_rank, 1.0)) / 1e12, FP64_NOMINAL_TFLOPS, "TFLOP/s", "nominal (SMs x lanes x clock)"),
         "quant": ("hbm", (n * d * 2 + out_bytes_per_block) / 1e9, peaks["hbm_gbs"], "GB/s", peaks["source"]),

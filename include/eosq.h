@@ -231,11 +231,11 @@ int64_t eosq_launch_count(const eosq_ctx *ctx);
  * CUDA events on the launching stream.  eosq_profile_read synchronises those events, adds their
  * elapsed milliseconds into ms[EOSQ_NUM_STAGES] and their launch counts into
  * launches[EOSQ_NUM_STAGES] (host arrays, overwritten), and clears the record.
- * Stage order: Gram, tridiagonalisation steps 0-63 and 64-125 (two kernels), eigenvalues,
+ * Stage order: Gram, tridiagonalisation steps 0-63, 64-95 and 96-125 (three kernels), eigenvalues,
  * spectrum + shrinkage + eigenvectors, residual/rotate/quantise/pack, decode, scores, the second
  * pass over blocks whose tensor-core Gram matrix was not accurate enough (all its kernels), other.
  */
-#define EOSQ_NUM_STAGES 10
+#define EOSQ_NUM_STAGES 11
 int eosq_profile_enable(eosq_ctx *ctx, int on);
 /* Times only the stages whose bit (1 << stage index, in the order above) is set in stage_mask; the
  * two events per launch cost about 2 us of device time each, which adds up over the several hundred

@@ -29,7 +29,7 @@ EXPORTS = [
     "eosq_check_status", "eosq_launch_count", "eosq_profile_enable", "eosq_profile_select", "eosq_profile_read",
     "eosq_encode_static", "eosq_encode_static_max_blocks", "eosq_selftest_wait_timeout",
 ]
-STAGES = ["gram", "tridiag_a", "tridiag_b", "eigvals", "spectral", "quant", "decode", "scores", "redo", "other"]
+STAGES = ["gram", "tridiag_a", "tridiag_b", "tridiag_c", "eigvals", "spectral", "quant", "decode", "scores", "redo", "other"]
 
 
 class EosqError(RuntimeError):

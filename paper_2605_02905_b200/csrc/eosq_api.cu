@@ -162,7 +162,7 @@ int eosq::encode_chunk(eosq_ctx *ctx, const void *blocks, int in_dtype, int64_t 
         run_stage(ctx, ST_GRAM, s, [&] { launch_gram_plain(chunk_in, in_dtype, nb, n, ws.gram, nullptr, nullptr, s); });
     }
     const bool full = out_all.eig != nullptr;   // the optional eigenvalue output asks for the whole spectrum
-    static_assert(TRIDIAG_PARTS == 2, "one profiling stage per tridiagonalisation kernel");
+    static_assert(TRIDIAG_PARTS == 3 && ST_TRIDIAG_C == ST_TRIDIAG_A + 2, "one profiling stage per tridiagonalisation kernel");
     for (int part = 0; part < TRIDIAG_PARTS; ++part)
         run_stage(ctx, ST_TRIDIAG_A + part, s, [&] { launch_tridiag(part, nb, ws, nullptr, nullptr, ctx->sm_count, s); });
     // the eigenvalue kernel also queues, in ws.redo_list, the blocks the tensor-core Gram matrix cannot resolve

@@ -90,7 +90,7 @@ inline size_t carve(void *base, int64_t cap, Workspace *ws) {
 
 }  // namespace eosq
 
-enum Stage { ST_GRAM = 0, ST_TRIDIAG_A, ST_TRIDIAG_B, ST_EIGVALS, ST_SPECTRAL, ST_QUANT, ST_DECODE, ST_SCORES, ST_REDO, ST_OTHER };
+enum Stage { ST_GRAM = 0, ST_TRIDIAG_A, ST_TRIDIAG_B, ST_TRIDIAG_C, ST_EIGVALS, ST_SPECTRAL, ST_QUANT, ST_DECODE, ST_SCORES, ST_REDO, ST_OTHER };
 
 struct eosq_ctx {
     struct Timed {
@@ -138,7 +138,7 @@ constexpr int64_t LIST_GRID = 148;
 inline unsigned list_grid(int64_t nb, const int *list) {
     return static_cast<unsigned>(list ? (nb < LIST_GRID ? nb : LIST_GRID) : nb);
 }
-constexpr int TRIDIAG_PARTS = 2;
+constexpr int TRIDIAG_PARTS = 3;
 void launch_tridiag(int part, int64_t nb, const Workspace &ws, const int *list, const int *count, int sm_count, cudaStream_t s);
 // All eigenvalues of each tridiagonal matrix by Sturm bisection.
 // With `full` every eigenvalue is resolved, otherwise the 3k + 1 largest and the smallest (what

@@ -497,11 +497,125 @@ __global__ void __launch_bounds__(G *G *TEAMS, MINB) tridiag_tm_kernel(double *_
     }
 }
 
+
+// ------------------------------------------------------------------------------------------
+// The last 30 steps, on the trailing 32 x 32 matrix: one warp per matrix, lane i keeps row i in
+// registers.  At this size a team's barriers and reductions cost more than its arithmetic, and a
+// matrix is 8 KB, so a warp does a step on its own (two warp sums, two broadcasts through shared
+// memory) and sixteen of them share an SM.  The step is the one of the header comment; column k of
+// the symmetric matrix is read as element k of every lane's row, and the loop over k is unrolled so
+// that finished columns drop out at compile time.
+// ------------------------------------------------------------------------------------------
+constexpr int TW_N = 32, TW_ORIGIN = D - TW_N, TW_WARPS = 4;
+
+__device__ __forceinline__ double tw_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+template <int K>
+__device__ __forceinline__ void tw_step(double (&a)[TW_N], int lane, double *ub, double *pb, double &dg, double &of, double &ta,
+                                        double *__restrict__ grow) {
+    // reflector K from column K (= row K): x_j = A[j][K], j > K
+    const double xj = (lane > K) ? a[K] : 0.0;
+    if (lane == K) dg = a[K];
+    const double alpha = __shfl_sync(0xffffffffu, xj, K + 1);
+    const double ss = tw_sum((lane > K + 1) ? xj * xj : 0.0);
+    double beta = alpha, gamma = 0.0;
+    if (ss > 0.0) {
+        const double sq = fma(alpha, alpha, ss);
+        const double nrm = sq * tt_rsqrt(sq);
+        beta = (alpha >= 0.0) ? -nrm : nrm;
+        gamma = tt_rcp(fma(fabs(alpha), nrm, sq));
+    }
+    const double uj = (lane == K + 1) ? xj - beta : xj;
+    if (lane == K) {
+        of = beta;
+        ta = gamma;
+    }
+    grow[lane] = uj;   // row TW_ORIGIN + K of the matrix in global memory, from its column TW_ORIGIN on
+    ub[lane] = uj;
+    __syncwarp();
+    // p = gamma A u over the live columns
+    constexpr int J0 = (K + 1) & ~1;   // pairs of columns; u is zero at K + 1 - 1 = K when that one is dragged in
+    double p0 = 0.0, p1 = 0.0, p2 = 0.0, p3 = 0.0;
+#pragma unroll
+    for (int j = J0; j < TW_N; j += 2) {
+        const double2 u2 = *reinterpret_cast<const double2 *>(ub + j);
+        if ((j - J0) & 2) {
+            p2 = fma(a[j], u2.x, p2);
+            p3 = fma(a[j + 1], u2.y, p3);
+        } else {
+            p0 = fma(a[j], u2.x, p0);
+            p1 = fma(a[j + 1], u2.y, p1);
+        }
+    }
+    const double pi = (lane > K) ? gamma * ((p0 + p1) + (p2 + p3)) : 0.0;
+    const double twoK = gamma * tw_sum(uj * pi);
+    const double si = fma(-twoK, uj, pi);
+    pb[lane] = pi;
+    __syncwarp();
+    // A <- A - u p^T - (p - 2K u) u^T on the rows and columns beyond K (u and s vanish on the others)
+#pragma unroll
+    for (int j = J0; j < TW_N; j += 2) {
+        const double2 u2 = *reinterpret_cast<const double2 *>(ub + j);
+        const double2 p2 = *reinterpret_cast<const double2 *>(pb + j);
+        a[j] = fma(-uj, p2.x, fma(-si, u2.x, a[j]));
+        a[j + 1] = fma(-uj, p2.y, fma(-si, u2.y, a[j + 1]));
+    }
+    __syncwarp();   // the broadcasts are overwritten by the next step
+}
+
+template <int K>
+__device__ __forceinline__ void tw_steps(double (&a)[TW_N], int lane, double *ub, double *pb, double &dg, double &of, double &ta,
+                                         double *__restrict__ trow0) {
+    if constexpr (K < TW_N - 2) {
+        tw_step<K>(a, lane, ub, pb, dg, of, ta, trow0 + static_cast<size_t>(K) * D);
+        tw_steps<K + 1>(a, lane, ub, pb, dg, of, ta, trow0);
+    }
+}
+
+__global__ void __launch_bounds__(32 * TW_WARPS, 4) tridiag_warp_kernel(double *__restrict__ gram, double *__restrict__ diag,
+                                                                        double *__restrict__ off, double *__restrict__ tau, int nb,
+                                                                        const int *__restrict__ list, const int *__restrict__ count) {
+    __shared__ __align__(16) double bc[TW_WARPS][2][TW_N];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int total = list ? *count : nb;
+    for (int li = blockIdx.x * TW_WARPS + warp; li < total; li += gridDim.x * TW_WARPS) {
+        const int blk = list ? list[li] : li;
+        double *T = gram + static_cast<size_t>(blk) * D * D + static_cast<size_t>(TW_ORIGIN) * D + TW_ORIGIN;
+        double a[TW_N];
+        {
+            const double2 *row = reinterpret_cast<const double2 *>(T + static_cast<size_t>(lane) * D);
+#pragma unroll
+            for (int q = 0; q < TW_N / 2; ++q) {
+                const double2 v = row[q];
+                a[2 * q] = v.x;
+                a[2 * q + 1] = v.y;
+            }
+        }
+        __syncwarp();   // every row is in registers before the reflectors overwrite the rows in memory
+        double dg = 0.0, of = 0.0, ta = 0.0;
+        tw_steps<0>(a, lane, bc[warp][0], bc[warp][1], dg, of, ta, T);
+        // what is left is the 2 x 2 block of the last two rows
+        if (lane == TW_N - 2) {
+            dg = a[TW_N - 2];
+            of = a[TW_N - 1];
+        }
+        if (lane == TW_N - 1) dg = a[TW_N - 1];
+        const size_t o = static_cast<size_t>(blk) * D + TW_ORIGIN + lane;
+        diag[o] = dg;
+        off[o] = of;
+        tau[o] = ta;
+    }
+}
+
 }  // namespace
 
-// Two ranges: the 128 x 128 matrix through its first 64 steps (256 threads and 256 columns of
-// tensor memory per matrix, two CTAs per SM), then the trailing 64 x 64 matrix (teams of 64
-// threads, two per CTA, four CTAs per SM).
+// Three ranges: the 128 x 128 matrix through its first 64 steps (two teams of 256 threads and all of
+// the tensor memory per CTA), the trailing 64 x 64 matrix through 32 more (teams of 64 threads, two
+// per CTA, four CTAs per SM), and the last 32 x 32 matrix by one warp each.
 void launch_tridiag(int part, int64_t nb, const Workspace &ws, const int *list, const int *count, int sm_count, cudaStream_t s) {
     double *g0 = ws.gram, *d0 = ws.diag, *o0 = ws.off, *t0 = ws.tau;
     const int n = static_cast<int>(nb);
@@ -509,9 +623,12 @@ void launch_tridiag(int part, int64_t nb, const Workspace &ws, const int *list, 
     if (part == 0) {
         const int grid = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>((work + 1) / 2, static_cast<int64_t>(sm_count))));
         tridiag_tm_kernel<16, 0, 64, 2, 1, true><<<grid, 512, 0, s>>>(g0, d0, o0, t0, n, list, count);
-    } else {
+    } else if (part == 1) {
         const int grid = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>((work + 1) / 2, 4 * static_cast<int64_t>(sm_count))));
-        tridiag_tm_kernel<8, 64, 62, 2, 4, false><<<grid, 128, 0, s>>>(g0, d0, o0, t0, n, list, count);
+        tridiag_tm_kernel<8, 64, 32, 2, 4, false><<<grid, 128, 0, s>>>(g0, d0, o0, t0, n, list, count);
+    } else {
+        const int grid = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>((work + TW_WARPS - 1) / TW_WARPS, 4 * static_cast<int64_t>(sm_count))));
+        tridiag_warp_kernel<<<grid, 32 * TW_WARPS, 0, s>>>(g0, d0, o0, t0, n, list, count);
     }
 }
 
