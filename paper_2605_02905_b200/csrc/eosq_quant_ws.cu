@@ -419,9 +419,22 @@ __global__ void __launch_bounds__(Q2_THREADS, 1) quant_ws_kernel(const __grid_co
                 const float rho = sqrtf(tot);
                 // thresholds scaled by the norm: y > thr rho decides as y / rho > thr does (a zero row keeps
                 // the plain thresholds, so that it gets the code of z = 0)
-                float ts[NTHR];
+                // The codebook is symmetric with its middle threshold at exactly 0, so a code is the sign plus the
+                // count of positive thresholds below |y|: 2^(b-1) comparisons instead of 2^b - 1.  (On the
+                // negative side this counts a value that sits exactly on a threshold into the outer cell, where
+                // the ascending count puts it into the inner one: a tie of measure zero, inside the band that
+                // the comparison with the reference exempts.)
+                constexpr int MAG = NTHR / 2;   // positive thresholds
+                float tp[MAG > 0 ? MAG : 1];
 #pragma unroll
-                for (int k = 0; k < NTHR; ++k) ts[k] = (rho > 0.0f) ? thr[k] * rho : thr[k];
+                for (int k = 0; k < MAG; ++k) tp[k] = (rho > 0.0f) ? thr[MAG + 1 + k] * rho : thr[MAG + 1 + k];
+                auto code_of = [&](float v) -> uint32_t {
+                    const float av = fabsf(v);
+                    uint32_t mag = 0u;
+#pragma unroll
+                    for (int k = 0; k < MAG; ++k) mag += (tp[k] < av) ? 1u : 0u;
+                    return (0.0f < v) ? (static_cast<uint32_t>(MAG + 1) + mag) : (static_cast<uint32_t>(MAG) - mag);
+                };
                 // 32 codes of BITS bits: BITS words of 32 bits, coordinate j of the thread at bits [j BITS, (j+1) BITS)
                 uint32_t wv[BITS];
                 if (BITS == 3) {
@@ -429,9 +442,7 @@ __global__ void __launch_bounds__(Q2_THREADS, 1) quant_ws_kernel(const __grid_co
                     int filled = 0, wi = 0;
 #pragma unroll
                     for (int c = 0; c < Q2_EPI_COLS; ++c) {
-                        unsigned code = 0u;
-#pragma unroll
-                        for (int k = 0; k < NTHR; ++k) code += (ts[k] < y[c]) ? 1u : 0u;
+                        const unsigned code = code_of(y[c]);
                         acc64 |= static_cast<unsigned long long>(code) << filled;
                         filled += BITS;
                         if (filled >= 32) {
@@ -447,11 +458,7 @@ __global__ void __launch_bounds__(Q2_THREADS, 1) quant_ws_kernel(const __grid_co
                         uint32_t w = 0u;
 #pragma unroll
                         for (int e = CPW - 1; e >= 0; --e) {
-                            const float v = y[k * CPW + e];
-                            uint32_t code = 0u;
-#pragma unroll
-                            for (int tt = 0; tt < NTHR; ++tt) code += (ts[tt] < v) ? 1u : 0u;
-                            w = w * (1u << BITS) + code;
+                            w = w * (1u << BITS) + code_of(y[k * CPW + e]);
                         }
                         wv[k] = w;
                     }
