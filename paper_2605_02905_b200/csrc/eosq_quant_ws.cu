@@ -451,6 +451,29 @@ __global__ void __launch_bounds__(Q2_THREADS, 1) quant_ws_kernel(const __grid_co
                             filled -= 32;
                         }
                     }
+                } else if (BITS == 2) {
+                    // Two bits: the three thresholds -t, 0, t are equally spaced, so the code is
+                    // floor(y / (t rho)) + 2 clamped to 0 .. 3.  One multiply-add rounded down onto
+                    // 1.5 2^23 + 2 leaves that integer in the low bits of the float, two min / max clamp it,
+                    // and a multiply-add per code packs the raw floats; their common offset leaves in one
+                    // subtraction per word.  (A value exactly on a threshold goes to the upper cell here
+                    // and to the lower one in the ascending count: measure zero, inside the exempted band;
+                    // a zero row, which is all ties, gets its codes directly.)
+                    constexpr float MAGIC = 12582912.0f;   // 1.5 2^23 = 0x4B400000: integers have an ulp of 1 there
+                    constexpr uint32_t MAGIC_BITS = 0x4B400000u;
+                    const float invt = (rho > 0.0f) ? __frcp_rn(thr[2] * rho) : 0.0f;
+#pragma unroll
+                    for (int k = 0; k < 2; ++k) {
+                        uint32_t w = 0u;
+#pragma unroll
+                        for (int e = 15; e >= 0; --e) {
+                            float f = __fmaf_rd(y[k * 16 + e], invt, MAGIC + 2.0f);
+                            f = fminf(fmaxf(f, MAGIC), MAGIC + 3.0f);
+                            w = w * 4u + __float_as_uint(f);
+                        }
+                        // sum of MAGIC_BITS 4^e over the sixteen codes, modulo 2^32
+                        wv[k] = (rho > 0.0f) ? w - MAGIC_BITS * 0x55555555u : 0x55555555u;
+                    }
                 } else {
                     constexpr int CPW = 32 / BITS;   // codes per 32-bit word, filled from the top code down
 #pragma unroll
